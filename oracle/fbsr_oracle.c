@@ -1,0 +1,372 @@
+/*
+ * Scalar CPU oracle for few-bit stochastic rounding (FBSR).
+ *
+ * TEST INFRASTRUCTURE ONLY.  One element at a time, no blocking, no vector
+ * code, no code shared with the CUDA library.  It exists so that the CUDA
+ * kernels can be compared with it bit for bit; nothing in the product path
+ * may call it.
+ *
+ * What it follows ("On Stochastic Rounding with Few Random Bits"):
+ *   Section II, Eq. (1)      value of a triple (s, e, t) in format (K, P, B; M)
+ *   Section II-A, Eq. (2)    exponent, clamped at 1-B so subnormals share one lsb
+ *   Section II-A, Eq. (3)    scaled significand sigma~ and delta~ = frac(sigma~)
+ *   Section II-A, Eq. (5)    sigma = floor(sigma~) + [R(delta~)], exponent
+ *                            incremented when sigma = 2^P
+ *   Section II-B             R_SRFF(d, n) = d + n 2^-N >= 1
+ *                            R_SRF (d, n) = d + (n + 1/2) 2^-N >= 1
+ *   Section III-F, Eq. (8)   R_SRC(d, n) = R_SRFF(Round(d 2^N) 2^-N, n), Round =
+ *                            nearest, ties to even
+ *
+ * The input is binary32, so delta~ is the rational r / 2^s with r, s integers.
+ * Each predicate is evaluated exactly by clearing denominators in 128-bit
+ * integers; there is no floating-point comparison anywhere in the rounding.
+ *
+ * Outside the paper (its Section II sets these aside): the magnitude is
+ * rounded and the sign copied; NaN -> quiet NaN with the sign kept; +-Inf ->
+ * +-Inf, or +-M if the format has none; finite |y| > M -> +-M; these elements
+ * are not SR-rounded and are excluded from the error sums.
+ *
+ * Random source (the paper leaves it open): Philox4x32-10, Salmon, Moraes,
+ * Dror, Shaw, "Parallel random numbers: as easy as 1, 2, 3", SC'11.
+ * Element with global index g and k bits per draw: dpw = 32 / k draws per
+ * word, E = 4 dpw elements per generator call, block b = g / E, counter
+ * (b lo, b hi, stream, 0), key (seed lo, seed hi), output word (g mod E) / dpw,
+ * field g mod dpw counted from the low bits.
+ *
+ * Build: gcc -O2 -std=c11 -ffp-contract=off -fno-fast-math -shared -fPIC
+ * (no contraction: every binary32 operation below rounds exactly once).
+ */
+#include <math.h>
+#include <stddef.h>
+#include <stdint.h>
+#include <string.h>
+
+typedef unsigned __int128 u128;
+
+enum { FMT_BF16 = 0, FMT_FP16 = 1, FMT_E4M3 = 2, FMT_E5M2 = 3 };
+enum { VAR_SRFF = 0, VAR_SRF = 1, VAR_SRC = 2 };
+enum { KIND_FINITE = 0, KIND_NAN = 1, KIND_INF = 2, KIND_SAT = 3 };
+
+typedef struct {
+    int K, P, B;
+    double M;          /* largest finite value */
+    uint32_t max_code; /* encoding of M */
+    int has_inf;
+    uint32_t inf_code;
+    uint32_t nan_code;
+} format_t;
+
+static const format_t FORMATS[4] = {
+    /* bf16 */ {16, 8, 127, 0x1.FEp127, 0x7F7Fu, 1, 0x7F80u, 0x7FC0u},
+    /* fp16 */ {16, 11, 15, 65504.0, 0x7BFFu, 1, 0x7C00u, 0x7E00u},
+    /* e4m3 */ {8, 4, 7, 448.0, 0x7Eu, 0, 0u, 0x7Fu},
+    /* e5m2 */ {8, 3, 15, 57344.0, 0x7Bu, 1, 0x7Cu, 0x7Fu},
+};
+
+typedef struct {
+    uint64_t n_finite, n_up, n_nan, n_inf, n_sat;
+    double sum_e, sum_e2, sum_signed_e, sum_abs_e;
+} oracle_stats_t;
+
+static uint32_t bits_of(float x) { uint32_t u; memcpy(&u, &x, 4); return u; }
+
+/* ------------------------------------------------------------------ Philox */
+void fbsr_oracle_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4])
+{
+    uint32_t c0 = ctr[0], c1 = ctr[1], c2 = ctr[2], c3 = ctr[3];
+    uint32_t k0 = key[0], k1 = key[1];
+    for (int round = 0; round < 10; ++round) {
+        uint64_t p0 = (uint64_t)0xD2511F53u * c0;
+        uint64_t p1 = (uint64_t)0xCD9E8D57u * c2;
+        uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ k0;
+        uint32_t n1 = (uint32_t)p1;
+        uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ k1;
+        uint32_t n3 = (uint32_t)p0;
+        c0 = n0; c1 = n1; c2 = n2; c3 = n3;
+        k0 += 0x9E3779B9u;
+        k1 += 0xBB67AE85u;
+    }
+    out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+uint32_t fbsr_oracle_draw(uint64_t seed, uint64_t g, int k, uint32_t stream)
+{
+    uint64_t dpw = 32u / (unsigned)k;
+    uint64_t E = 4 * dpw;
+    uint64_t b = g / E;
+    uint32_t ctr[4] = {(uint32_t)b, (uint32_t)(b >> 32), stream, 0u};
+    uint32_t key[2] = {(uint32_t)seed, (uint32_t)(seed >> 32)};
+    uint32_t out[4];
+    fbsr_oracle_philox4x32_10(ctr, key, out);
+    uint64_t w = (g % E) / dpw;
+    uint64_t j = g % dpw;
+    return (out[w] >> (j * (unsigned)k)) & ((1u << k) - 1u);
+}
+
+/* The packed word stream itself: word index W (global) is output W mod 4 of
+ * block W / 4.  Element g reads field g mod dpw of word g / dpw. */
+void fbsr_oracle_random_words(uint64_t seed, uint64_t first_word, size_t nwords, uint32_t stream,
+                              uint32_t* out_words)
+{
+    for (size_t j = 0; j < nwords; ++j) {
+        uint64_t W = first_word + j, b = W / 4;
+        uint32_t ctr[4] = {(uint32_t)b, (uint32_t)(b >> 32), stream, 0u};
+        uint32_t key[2] = {(uint32_t)seed, (uint32_t)(seed >> 32)};
+        uint32_t out[4];
+        fbsr_oracle_philox4x32_10(ctr, key, out);
+        out_words[j] = out[W % 4];
+    }
+}
+
+static uint32_t field_of_words(const uint32_t* words, size_t i, int k)
+{
+    size_t dpw = 32u / (unsigned)k;
+    return (words[i / dpw] >> ((i % dpw) * (unsigned)k)) & ((1u << k) - 1u);
+}
+
+/* ------------------------------------------------------------- Eq. (1) */
+float fbsr_oracle_decode(int fmt, uint32_t code)
+{
+    const format_t* f = &FORMATS[fmt];
+    uint32_t s = (code >> (f->K - 1)) & 1u;
+    uint32_t e = (code >> (f->P - 1)) & ((1u << (f->K - f->P)) - 1u);
+    uint32_t t = code & ((1u << (f->P - 1)) - 1u);
+    uint32_t mag = code & ((1u << (f->K - 1)) - 1u);
+    double v;
+    if (f->has_inf && mag == f->inf_code) v = INFINITY;
+    else if ((f->has_inf && mag > f->inf_code) || (!f->has_inf && mag == f->nan_code)) v = NAN;
+    else if (e == 0) v = ldexp(0.0 + ldexp((double)t, 1 - f->P), 1 - f->B);
+    else v = ldexp(1.0 + ldexp((double)t, 1 - f->P), (int)e - f->B);
+    float r = (float)v; /* exact: every target value is a binary32 value */
+    return s ? -r : r;
+}
+
+/* ------------------------------------------------ one element, Eq. (2)-(8) */
+uint32_t fbsr_oracle_round_one(float y, int fmt, int variant, int N, uint32_t n,
+                               int* kind_out, int* up_out, double* delta_out)
+{
+    const format_t* f = &FORMATS[fmt];
+    const int P = f->P, B = f->B;
+    uint32_t yb = bits_of(y);
+    uint32_t sign = (yb >> 31) << (f->K - 1);
+    uint32_t mag = yb & 0x7FFFFFFFu;
+    int kind = KIND_FINITE, up = 0;
+    double delta = 0.0;
+    uint32_t code;
+
+    if (mag > 0x7F800000u) { kind = KIND_NAN; code = f->nan_code; goto done; }
+    if (mag == 0x7F800000u) { kind = KIND_INF; code = f->has_inf ? f->inf_code : f->max_code; goto done; }
+    if (mag == 0u) { code = 0u; goto done; }
+    if ((double)fabsf(y) > f->M) { kind = KIND_SAT; code = f->max_code; goto done; }
+
+    {
+        /* |y| = m * 2^q exactly, m the 24-bit integer significand. */
+        uint32_t e32 = mag >> 23, t32 = mag & 0x7FFFFFu;
+        uint64_t m = e32 ? (t32 | 0x800000u) : t32;
+        int q = (e32 ? (int)e32 : 1) - 150;
+        /* floor(log2 |y|) */
+        int msb = 63 - __builtin_clzll(m);
+        int flog = msb + q;
+        int e = flog > 1 - B ? flog : 1 - B;          /* Eq. (2) */
+        /* sigma~ = |y| 2^-e 2^(P-1) = m / 2^s,  s = e - q - (P-1) > 0.  Eq. (3) */
+        int s = e - q - (P - 1);
+        uint64_t fl, r;
+        if (s >= 64) {
+            /* m < 2^24 so delta~ < 2^-40: with N <= 16 no predicate can hold
+               (delta~ + (n + 1/2) 2^-N <= 2^-40 + 1 - 2^-17 < 1; Round(delta~ 2^N) = 0). */
+            fl = 0; r = m; up = 0;
+            delta = ldexp((double)m, -s);
+        } else {
+            fl = m >> s;
+            r = m & (((uint64_t)1 << s) - 1u);
+            delta = ldexp((double)r, -s);            /* exact */
+            u128 one = (u128)1;
+            if (variant == VAR_SRFF) {
+                /* r/2^s + n/2^N >= 1   <=>   r 2^N + n 2^s >= 2^(s+N) */
+                up = ((u128)r << N) + ((u128)n << s) >= (one << (s + N));
+            } else if (variant == VAR_SRF) {
+                /* r/2^s + (2n+1)/2^(N+1) >= 1 */
+                up = ((u128)r << (N + 1)) + ((u128)(2u * n + 1u) << s) >= (one << (s + N + 1));
+            } else {
+                /* qn = Round(r 2^N / 2^s), nearest, ties to even; then qn + n >= 2^N */
+                u128 num = (u128)r << N;
+                u128 qn = num >> s;
+                u128 rem = num - (qn << s);
+                u128 twice = rem << 1, den = one << s;
+                if (twice > den || (twice == den && (qn & 1u))) qn += 1;
+                up = qn + n >= (one << N);
+            }
+        }
+        uint64_t sigma = fl + (uint64_t)up;            /* Eq. (5) */
+        if (sigma == ((uint64_t)1 << P)) { sigma >>= 1; e += 1; }
+        uint32_t be, t;
+        if (sigma >= ((uint64_t)1 << (P - 1))) { be = (uint32_t)(e + B); t = (uint32_t)(sigma - ((uint64_t)1 << (P - 1))); }
+        else { be = 0u; t = (uint32_t)sigma; }
+        code = (be << (P - 1)) | t;
+    }
+done:
+    if (kind_out) *kind_out = kind;
+    if (up_out) *up_out = up;
+    if (delta_out) *delta_out = delta;
+    return sign | code;
+}
+
+static void store_code(void* dst, size_t i, int fmt, uint32_t code)
+{
+    if (FORMATS[fmt].K == 16) ((uint16_t*)dst)[i] = (uint16_t)code;
+    else ((uint8_t*)dst)[i] = (uint8_t)code;
+}
+
+static uint32_t load_code(const void* src, size_t i, int fmt)
+{
+    return FORMATS[fmt].K == 16 ? ((const uint16_t*)src)[i] : ((const uint8_t*)src)[i];
+}
+
+/* y = fl32(x * scale), one rounded binary32 multiply (scaled tensors,
+ * Section I-A).  A NaN input is passed through untouched so that its sign,
+ * which the output keeps, does not depend on how a platform propagates NaNs. */
+static float scaled(float x, float scale) { return isnan(x) ? x : x * scale; }
+
+/* NaNs produced by arithmetic (optimizer, accumulation) have a platform
+ * dependent sign; they are written as the positive quiet NaN. */
+static float arith_result(float y) { return isnan(y) ? NAN : y; }
+
+static int bad_args(int fmt, int variant, int k)
+{
+    return fmt < 0 || fmt > 3 || variant < 0 || variant > 2 || k < 1 || k > 16;
+}
+
+/* ------------------------------------------------------------ array forms */
+int fbsr_oracle_round(const float* src, void* dst, size_t n, int fmt, int variant, int k,
+                      uint64_t seed, uint64_t offset, float scale)
+{
+    if (bad_args(fmt, variant, k)) return 1;
+    for (size_t i = 0; i < n; ++i) {
+        float y = scaled(src[i], scale);
+        uint32_t nr = fbsr_oracle_draw(seed, offset + i, k, 0u);
+        store_code(dst, i, fmt, fbsr_oracle_round_one(y, fmt, variant, k, nr, 0, 0, 0));
+    }
+    return 0;
+}
+
+int fbsr_oracle_round_bits(const float* src, void* dst, size_t n, int fmt, int variant, int k,
+                           const uint32_t* rand_words, float scale)
+{
+    if (bad_args(fmt, variant, k)) return 1;
+    for (size_t i = 0; i < n; ++i) {
+        float y = scaled(src[i], scale);
+        uint32_t nr = field_of_words(rand_words, i, k);
+        store_code(dst, i, fmt, fbsr_oracle_round_one(y, fmt, variant, k, nr, 0, 0, 0));
+    }
+    return 0;
+}
+
+/* Error of one SR-rounded element in target ulps: e = up - delta~ (the
+ * quantity whose mean Section III calls bias).  Group g holds elements
+ * [g*group_size, (g+1)*group_size) of this call. */
+int fbsr_oracle_round_stats(const float* src, void* dst, size_t n, int fmt, int variant, int k,
+                            uint64_t seed, uint64_t offset, float scale, size_t group_size,
+                            double* group_sum_e, double* group_sum_e2, oracle_stats_t* total)
+{
+    if (bad_args(fmt, variant, k)) return 1;
+    long double se = 0, se2 = 0, sse = 0, sae = 0, ge = 0, ge2 = 0;
+    oracle_stats_t st;
+    memset(&st, 0, sizeof st);
+    for (size_t i = 0; i < n; ++i) {
+        float y = scaled(src[i], scale);
+        uint32_t nr = fbsr_oracle_draw(seed, offset + i, k, 0u);
+        int kind, up;
+        double delta;
+        store_code(dst, i, fmt, fbsr_oracle_round_one(y, fmt, variant, k, nr, &kind, &up, &delta));
+        if (kind == KIND_FINITE) {
+            double e = (double)up - delta;
+            st.n_finite++;
+            st.n_up += (uint64_t)up;
+            se += e; se2 += e * e;
+            sse += signbit(y) ? -e : e;
+            sae += fabs(e);
+            ge += e; ge2 += e * e;
+        } else if (kind == KIND_NAN) st.n_nan++;
+        else if (kind == KIND_INF) st.n_inf++;
+        else st.n_sat++;
+        if (group_size && ((i + 1) % group_size == 0 || i + 1 == n)) {
+            size_t g = i / group_size;
+            if (group_sum_e) group_sum_e[g] = (double)ge;
+            if (group_sum_e2) group_sum_e2[g] = (double)ge2;
+            ge = 0; ge2 = 0;
+        }
+    }
+    st.sum_e = (double)se; st.sum_e2 = (double)se2;
+    st.sum_signed_e = (double)sse; st.sum_abs_e = (double)sae;
+    if (total) *total = st;
+    return 0;
+}
+
+/* Fused optimizer steps.  Algorithm 1 only says: compute the update in the
+ * wide format, then SR-round the new weight.  The binary32 operation list is
+ * this library's own definition; each line is one correctly rounded operation
+ * (fmaf = fused multiply-add). */
+int fbsr_oracle_sgd_update(float* w, const float* g, float* m, void* dst, size_t n, int fmt,
+                           int variant, int k, uint64_t seed, uint64_t offset, float lr, float mu)
+{
+    if (bad_args(fmt, variant, k)) return 1;
+    for (size_t i = 0; i < n; ++i) {
+        float m2 = fmaf(mu, m[i], g[i]);
+        float w2 = fmaf(-lr, m2, w[i]);
+        m[i] = m2; w[i] = w2;
+        uint32_t nr = fbsr_oracle_draw(seed, offset + i, k, 0u);
+        store_code(dst, i, fmt, fbsr_oracle_round_one(arith_result(w2), fmt, variant, k, nr, 0, 0, 0));
+    }
+    return 0;
+}
+
+void fbsr_oracle_adam_coefficients(float lr, float beta1, float beta2, int step, float out[4])
+{
+    double b1t = 1.0, b2t = 1.0;
+    for (int t = 0; t < step; ++t) { b1t *= (double)beta1; b2t *= (double)beta2; }
+    out[0] = (float)((double)lr / (1.0 - b1t));
+    out[1] = (float)(1.0 / sqrt(1.0 - b2t));
+    out[2] = (float)(1.0 - (double)beta1);
+    out[3] = (float)(1.0 - (double)beta2);
+}
+
+int fbsr_oracle_adam_update(float* w, const float* g, float* m, float* v, void* dst, size_t n,
+                            int fmt, int variant, int k, uint64_t seed, uint64_t offset,
+                            float lr, float beta1, float beta2, float eps, int step)
+{
+    if (bad_args(fmt, variant, k) || step < 1) return 1;
+    float c[4];
+    fbsr_oracle_adam_coefficients(lr, beta1, beta2, step, c);
+    const float c1 = c[0], c2 = c[1], a1 = c[2], a2 = c[3];
+    for (size_t i = 0; i < n; ++i) {
+        float a1g = a1 * g[i];
+        float m2 = fmaf(beta1, m[i], a1g);
+        float a2g = a2 * g[i];
+        float a2gg = a2g * g[i];
+        float v2 = fmaf(beta2, v[i], a2gg);
+        float sq = sqrtf(v2);
+        float sc = sq * c2;
+        float d = sc + eps;
+        float qt = m2 / d;
+        float w2 = fmaf(-c1, qt, w[i]);
+        m[i] = m2; v[i] = v2; w[i] = w2;
+        uint32_t nr = fbsr_oracle_draw(seed, offset + i, k, 0u);
+        store_code(dst, i, fmt, fbsr_oracle_round_one(arith_result(w2), fmt, variant, k, nr, 0, 0, 0));
+    }
+    return 0;
+}
+
+/* Low-precision accumulation (last line of Algorithm 1): the stored weight is
+ * widened exactly, the update added in binary32, the sum SR-rounded back. */
+int fbsr_oracle_accumulate(void* w_lp, const float* update, size_t n, int fmt, int variant, int k,
+                           uint64_t seed, uint64_t offset)
+{
+    if (bad_args(fmt, variant, k)) return 1;
+    for (size_t i = 0; i < n; ++i) {
+        float wv = fbsr_oracle_decode(fmt, load_code(w_lp, i, fmt));
+        float y = arith_result(wv + update[i]);
+        uint32_t nr = fbsr_oracle_draw(seed, offset + i, k, 0u);
+        store_code(w_lp, i, fmt, fbsr_oracle_round_one(y, fmt, variant, k, nr, 0, 0, 0));
+    }
+    return 0;
+}
