@@ -1,0 +1,173 @@
+/*
+ * fbsr.h -- few-bit stochastic rounding (FBSR) on NVIDIA B200 (sm_100a).
+ *
+ * C-ABI of libfbsr.so.  The operations follow "On Stochastic Rounding with Few
+ * Random Bits" (Fitzgibbon & Felix): a binary32 value y is rounded to a narrower
+ * format (K, P, B; M) by
+ *     e~     = max(floor(log2 |y|), 1 - B)                      Section II-A, Eq. (2)
+ *     sigma~ = |y| 2^-e~ 2^(P-1),  delta~ = sigma~ - floor(sigma~)           Eq. (3)
+ *     sigma  = floor(sigma~) + [R(delta~, n)]                                Eq. (5)
+ * with n an integer of N = k_bits random bits and R one of
+ *     R_SRFF(d, n) = d + n 2^-N >= 1                            Section II-B
+ *     R_SRF (d, n) = d + (n + 1/2) 2^-N >= 1                    Section II-B
+ *     R_SRC (d, n) = R_SRFF(Round(d 2^N) 2^-N, n)               Section III-F, Eq. (8)
+ * (Round = nearest, ties to even).  sigma = 2^P increments the exponent.
+ *
+ * Conventions shared by every entry point unless stated otherwise
+ *   - Pointers are DEVICE pointers owned by the caller.  The library allocates no
+ *     memory, never synchronises, and only enqueues work on `cuda_stream`
+ *     (a cudaStream_t passed as void*; NULL = the default stream) of the current
+ *     device.  Buffers must stay valid until that work has run.
+ *   - Results are a pure function of the arguments: the same (seed, offset)
+ *     gives the same bits on every call and for every way of splitting a tensor
+ *     into calls, provided `offset` is the global index of element 0.
+ *   - The magnitude is rounded and the sign copied.  NaN -> quiet NaN, sign of
+ *     the input kept (0x7FC0 bf16, 0x7E00 fp16, 0x7F e4m3 and e5m2).  +-Inf ->
+ *     +-Inf, or +-M for e4m3, which has no infinity.  Finite |y| > M -> +-M.
+ *     None of these consume the paper's predicates (Section II leaves values
+ *     outside the finite range to deterministic rounding).
+ *   - Random draws: Philox4x32-10 with key (seed lo, seed hi).  With
+ *     dpw = 32 / k_bits (integer division) draws per 32-bit word and E = 4 dpw,
+ *     the element with global index g uses field (g mod dpw), low bits first, of
+ *     output word ((g mod E) / dpw) of the generator call with counter
+ *     (b lo, b hi, 0, 0), b = g / E.  The paper leaves the generator open
+ *     (Section II-B); this indexing is the library's definition.
+ *   - Any n (including 0) and any element alignment are accepted.  The fast
+ *     path needs src 32-byte aligned, dst 16-byte aligned and `offset` a multiple
+ *     of the tile size reported by fbsr_tile_elements(); other calls are served
+ *     by a slower kernel with identical results.
+ *   - Errors are reported by the return value only.  Nothing is written on error.
+ */
+#ifndef FBSR_H
+#define FBSR_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    FBSR_OK = 0,
+    FBSR_ERR_INVALID_ARG = 1, /* null pointer with n > 0, bad enum, k_bits outside 1..16, bad scale */
+    FBSR_ERR_UNSUPPORTED = 2, /* a combination this build does not implement */
+    FBSR_ERR_ALIGNMENT = 3,   /* a pointer is not aligned to its element size */
+    FBSR_ERR_CUDA = 4,        /* the CUDA runtime reported an error at launch */
+    FBSR_ERR_WORKSPACE = 5    /* workspace missing or too small */
+} fbsr_status;
+
+/* Target formats (K, P, B; M), Section II.  P counts the hidden bit. */
+typedef enum {
+    FBSR_BF16 = 0, /* (16,  8, 127; 0x1.FEp127) */
+    FBSR_FP16 = 1, /* (16, 11,  15; 65504)      */
+    FBSR_E4M3 = 2, /* ( 8,  4,   7; 448)   OCP E4M3: no Inf, S.1111.111 is NaN */
+    FBSR_E5M2 = 3  /* ( 8,  3,  15; 57344) */
+} fbsr_fmt;
+
+/* Round-up predicates, Section II-B and Eq. (8). */
+typedef enum { FBSR_SRFF = 0, FBSR_SRF = 1, FBSR_SRC = 2 } fbsr_variant;
+
+/* Error statistics over the SR-rounded elements of one call.  e = up - delta~
+ * is the rounding error of the magnitude in target ulps, the quantity whose
+ * mean Section III calls bias.  NaN, Inf and saturated elements are counted
+ * but excluded from the sums. */
+typedef struct {
+    uint64_t n_finite;   /* elements that were SR-rounded (|y| <= M, zeros included) */
+    uint64_t n_up;       /* of those, how many rounded up in magnitude */
+    uint64_t n_nan;
+    uint64_t n_inf;
+    uint64_t n_sat;      /* finite |y| > M */
+    double sum_e;        /* sum of e */
+    double sum_e2;       /* sum of e^2 */
+    double sum_signed_e; /* sum of sign(y) e: error of the signed value */
+    double sum_abs_e;    /* sum of |e| */
+} fbsr_stats;
+
+/* ---------------------------------------------------------------------------
+ * fbsr_round -- Section II-A/II-B/III-F: dst[i] = FBSR(fl32(src[i] * scale)).
+ *   src      device, n binary32 values (read only; must not overlap dst)
+ *   dst      device, n codes: uint16 for bf16/fp16, uint8 for e4m3/e5m2
+ *   fmt, variant, k_bits   fbsr_fmt, fbsr_variant, N in 1..16
+ *   seed, offset           Philox key and global index of element 0
+ *   scale    finite, > 0; the per-tensor factor of a scaled tensor (Section I-A),
+ *            applied as one rounded binary32 multiply
+ * ------------------------------------------------------------------------- */
+int fbsr_round(const float* src, void* dst, size_t n, int fmt, int variant, int k_bits,
+               uint64_t seed, uint64_t offset, float scale, void* cuda_stream);
+
+/* fbsr_round_bits -- the same rounding with caller-supplied random bits
+ * (Section II-B: "random numbers will be supplied as a finite sequence of random
+ * bits").  rand_words: device, ceil(n / dpw) words; element i uses field
+ * (i mod dpw) of word (i / dpw), low bits first; higher bits are ignored. */
+int fbsr_round_bits(const float* src, void* dst, size_t n, int fmt, int variant, int k_bits,
+                    const uint32_t* rand_words, float scale, void* cuda_stream);
+
+/* fbsr_round_stats -- fbsr_round plus the error statistics of Section III
+ * (bias = mean of e) accumulated in binary64.
+ *   group_size       0, or the length of the consecutive groups of this call's
+ *                    elements (group j = elements [j group_size, (j+1) group_size))
+ *   group_sum_e/_e2  device, ceil(n / group_size) doubles each, overwritten with
+ *                    the per-group sums of e and e^2; may be NULL when group_size = 0.
+ *                    Group sums are added with atomics: their last bits may vary
+ *                    from run to run.
+ *   total            device, one fbsr_stats, overwritten.  Totals are reduced in a
+ *                    fixed order and are reproducible bit for bit.
+ *   workspace        device scratch of at least fbsr_stats_workspace_bytes() bytes,
+ *                    8-byte aligned; contents on entry are ignored. */
+size_t fbsr_stats_workspace_bytes(void);
+int fbsr_round_stats(const float* src, void* dst, size_t n, int fmt, int variant, int k_bits,
+                     uint64_t seed, uint64_t offset, float scale, size_t group_size,
+                     double* group_sum_e, double* group_sum_e2, fbsr_stats* total,
+                     void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* fbsr_sgd_update -- last line of Algorithm 1 with a binary32 master copy:
+ *     m' = fma(mu, m, g);  w' = fma(-lr, m', w);  dst = FBSR(w')
+ * master_w and momentum are updated in place; grad is read only.  Every
+ * operation is one correctly rounded binary32 operation (no flush to zero). */
+int fbsr_sgd_update(float* master_w, const float* grad, float* momentum, void* dst_lp, size_t n,
+                    int fmt, int variant, int k_bits, uint64_t seed, uint64_t offset,
+                    float lr, float mu, void* cuda_stream);
+
+/* fbsr_adam_update -- same, with Adam (no weight decay).  Host scalars, in
+ * binary64 then rounded to binary32: b1t = beta1^step and b2t = beta2^step by
+ * repeated multiplication, c1 = lr / (1 - b1t), c2 = 1 / sqrt(1 - b2t),
+ * a1 = 1 - beta1, a2 = 1 - beta2.  Per element, binary32:
+ *     m' = fma(beta1, m, a1 g);  v' = fma(beta2, v, (a2 g) g);
+ *     d  = sqrt(v') c2 + eps;    w' = fma(-c1, m' / d, w);  dst = FBSR(w')
+ * step >= 1 is the 1-based step count. */
+int fbsr_adam_update(float* master_w, const float* grad, float* m, float* v, void* dst_lp, size_t n,
+                     int fmt, int variant, int k_bits, uint64_t seed, uint64_t offset,
+                     float lr, float beta1, float beta2, float eps, int step, void* cuda_stream);
+
+/* fbsr_accumulate -- Algorithm 1, "w8 <- RoundTo8(w16 + u16)" with the sum
+ * formed in binary32:  w_lp[i] = FBSR(fl32(value(w_lp[i]) + update[i])), in place.
+ * A NaN sum is written as the positive quiet NaN. */
+int fbsr_accumulate(void* w_lp, const float* update, size_t n, int fmt, int variant, int k_bits,
+                    uint64_t seed, uint64_t offset, void* cuda_stream);
+
+/* fbsr_round_host -- fbsr_round for HOST buffers (pinned memory gives overlap):
+ * copies src to the device in chunks, rounds, copies the codes back, using
+ * dev_workspace (device, >= fbsr_round_host_min_workspace() bytes, 256-byte
+ * aligned) as a double buffer.  Work is enqueued on cuda_stream and on an
+ * internal copy stream that is joined back into cuda_stream before return;
+ * dst_host is valid once cuda_stream has been synchronised. */
+size_t fbsr_round_host_min_workspace(void);
+int fbsr_round_host(const float* src_host, void* dst_host, size_t n, int fmt, int variant, int k_bits,
+                    uint64_t seed, uint64_t offset, float scale, void* dev_workspace,
+                    size_t workspace_bytes, void* cuda_stream);
+
+/* Elements per warp tile of the fast path for k_bits: `offset` values that are
+ * multiples of it keep a sharded call on the fast path.  0 if k_bits is invalid. */
+size_t fbsr_tile_elements(int k_bits);
+
+/* Number of kernel launches the library has enqueued since it was loaded. */
+uint64_t fbsr_launch_count(void);
+
+const char* fbsr_status_string(int status);
+int fbsr_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FBSR_H */

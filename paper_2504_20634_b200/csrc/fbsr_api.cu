@@ -1,0 +1,255 @@
+// C-ABI entry points of libfbsr.so: argument validation, host-side scalars, dispatch by format,
+// and the chunked host-buffer pipeline.  See include/fbsr.h for the contract of each call.
+#include <atomic>
+#include <cmath>
+#include <mutex>
+
+#include "../../include/fbsr.h"
+#include "fbsr_internal.h"
+
+namespace fbsr {
+
+static std::atomic<uint64_t> g_launches{0};
+void count_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
+
+int sm_count()
+{
+    static int cached[64] = {0};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+    if (cached[dev] == 0) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) n = 148;
+        cached[dev] = n;
+    }
+    return cached[dev];
+}
+
+namespace {
+
+typedef int (*dispatch_fn)(const CallArgs&);
+const dispatch_fn kRound[4] = {dispatch_round_0, dispatch_round_1, dispatch_round_2, dispatch_round_3};
+const dispatch_fn kOptim[4] = {dispatch_optim_0, dispatch_optim_1, dispatch_optim_2, dispatch_optim_3};
+
+inline bool bad_enum(int fmt, int variant, int k) { return fmt < 0 || fmt > 3 || variant < 0 || variant > 2 || k < 1 || k > 16; }
+inline size_t code_bytes(int fmt) { return fmt <= 1 ? 2 : 1; }
+inline bool misaligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) != 0; }
+
+inline int finish(int rc)
+{
+    if (rc != 0) return FBSR_ERR_UNSUPPORTED;
+    return cudaGetLastError() == cudaSuccess ? FBSR_OK : FBSR_ERR_CUDA;
+}
+
+CallArgs base_args(OpKind op, int variant, int k, size_t n, uint64_t seed, uint64_t offset, void* dst, void* stream)
+{
+    CallArgs a{};
+    a.op = op; a.variant = variant; a.k = k; a.n = n; a.seed = seed; a.offset = offset;
+    a.dst = dst; a.stream = static_cast<cudaStream_t>(stream); a.scale = 1.0f;
+    return a;
+}
+
+int check_round(const float* src, const void* dst, size_t n, int fmt, int variant, int k, float scale)
+{
+    if (bad_enum(fmt, variant, k)) return FBSR_ERR_INVALID_ARG;
+    if (!(scale > 0.0f) || !std::isfinite(scale)) return FBSR_ERR_INVALID_ARG;
+    if (n > 0 && (src == nullptr || dst == nullptr)) return FBSR_ERR_INVALID_ARG;
+    if (misaligned(src, 4) || misaligned(dst, code_bytes(fmt))) return FBSR_ERR_ALIGNMENT;
+    return FBSR_OK;
+}
+
+}  // namespace
+}  // namespace fbsr
+
+using namespace fbsr;
+
+extern "C" {
+
+int fbsr_round(const float* src, void* dst, size_t n, int fmt, int variant, int k_bits, uint64_t seed,
+               uint64_t offset, float scale, void* cuda_stream)
+{
+    if (int rc = check_round(src, dst, n, fmt, variant, k_bits, scale)) return rc;
+    if (n == 0) return FBSR_OK;
+    CallArgs a = base_args(OP_ROUND, variant, k_bits, n, seed, offset, dst, cuda_stream);
+    a.src = src; a.scale = scale;
+    return finish(kRound[fmt](a));
+}
+
+int fbsr_round_bits(const float* src, void* dst, size_t n, int fmt, int variant, int k_bits,
+                    const uint32_t* rand_words, float scale, void* cuda_stream)
+{
+    if (int rc = check_round(src, dst, n, fmt, variant, k_bits, scale)) return rc;
+    if (n > 0 && rand_words == nullptr) return FBSR_ERR_INVALID_ARG;
+    if (misaligned(rand_words, 4)) return FBSR_ERR_ALIGNMENT;
+    if (n == 0) return FBSR_OK;
+    CallArgs a = base_args(OP_ROUND_BITS, variant, k_bits, n, 0, 0, dst, cuda_stream);
+    a.src = src; a.scale = scale; a.words = rand_words;
+    return finish(kRound[fmt](a));
+}
+
+size_t fbsr_stats_workspace_bytes(void) { return (size_t)MAX_SLOW_GRID * sizeof(fbsr_stats); }
+
+int fbsr_round_stats(const float* src, void* dst, size_t n, int fmt, int variant, int k_bits, uint64_t seed,
+                     uint64_t offset, float scale, size_t group_size, double* group_sum_e, double* group_sum_e2,
+                     fbsr_stats* total, void* workspace, size_t workspace_bytes, void* cuda_stream)
+{
+    if (int rc = check_round(src, dst, n, fmt, variant, k_bits, scale)) return rc;
+    if (total == nullptr) return FBSR_ERR_INVALID_ARG;
+    if (group_size > 0 && n > 0 && (group_sum_e == nullptr || group_sum_e2 == nullptr)) return FBSR_ERR_INVALID_ARG;
+    if (misaligned(total, 8) || misaligned(group_sum_e, 8) || misaligned(group_sum_e2, 8)) return FBSR_ERR_ALIGNMENT;
+    if (workspace == nullptr || workspace_bytes < fbsr_stats_workspace_bytes()) return FBSR_ERR_WORKSPACE;
+    if (misaligned(workspace, 8)) return FBSR_ERR_ALIGNMENT;
+    CallArgs a = base_args(OP_ROUND_STATS, variant, k_bits, n, seed, offset, dst, cuda_stream);
+    a.src = src; a.scale = scale; a.group_size = group_size;
+    a.gsum_e = group_sum_e; a.gsum_e2 = group_sum_e2; a.total = total; a.partials = workspace;
+    if (group_size > 0 && n > 0) {
+        const size_t groups = (n + group_size - 1) / group_size;
+        if (cudaMemsetAsync(group_sum_e, 0, groups * sizeof(double), a.stream) != cudaSuccess ||
+            cudaMemsetAsync(group_sum_e2, 0, groups * sizeof(double), a.stream) != cudaSuccess)
+            return FBSR_ERR_CUDA;
+    }
+    return finish(kRound[fmt](a));
+}
+
+int fbsr_sgd_update(float* master_w, const float* grad, float* momentum, void* dst_lp, size_t n, int fmt,
+                    int variant, int k_bits, uint64_t seed, uint64_t offset, float lr, float mu, void* cuda_stream)
+{
+    if (bad_enum(fmt, variant, k_bits)) return FBSR_ERR_INVALID_ARG;
+    if (n > 0 && (!master_w || !grad || !momentum || !dst_lp)) return FBSR_ERR_INVALID_ARG;
+    if (misaligned(master_w, 4) || misaligned(grad, 4) || misaligned(momentum, 4) ||
+        misaligned(dst_lp, code_bytes(fmt))) return FBSR_ERR_ALIGNMENT;
+    if (n == 0) return FBSR_OK;
+    CallArgs a = base_args(OP_SGD, variant, k_bits, n, seed, offset, dst_lp, cuda_stream);
+    a.w = master_w; a.g = grad; a.m = momentum; a.neg_lr = -lr; a.mu = mu;
+    return finish(kOptim[fmt](a));
+}
+
+int fbsr_adam_update(float* master_w, const float* grad, float* m, float* v, void* dst_lp, size_t n, int fmt,
+                     int variant, int k_bits, uint64_t seed, uint64_t offset, float lr, float beta1, float beta2,
+                     float eps, int step, void* cuda_stream)
+{
+    if (bad_enum(fmt, variant, k_bits) || step < 1) return FBSR_ERR_INVALID_ARG;
+    if (n > 0 && (!master_w || !grad || !m || !v || !dst_lp)) return FBSR_ERR_INVALID_ARG;
+    if (misaligned(master_w, 4) || misaligned(grad, 4) || misaligned(m, 4) || misaligned(v, 4) ||
+        misaligned(dst_lp, code_bytes(fmt))) return FBSR_ERR_ALIGNMENT;
+    if (n == 0) return FBSR_OK;
+    // Bias-correction scalars in binary64, rounded once to binary32.
+    double b1t = 1.0, b2t = 1.0;
+    for (int t = 0; t < step; ++t) { b1t *= (double)beta1; b2t *= (double)beta2; }
+    CallArgs a = base_args(OP_ADAM, variant, k_bits, n, seed, offset, dst_lp, cuda_stream);
+    a.w = master_w; a.g = grad; a.m = m; a.v = v;
+    a.beta1 = beta1; a.beta2 = beta2; a.eps = eps;
+    a.neg_c1 = -(float)((double)lr / (1.0 - b1t));
+    a.c2 = (float)(1.0 / std::sqrt(1.0 - b2t));
+    a.a1 = (float)(1.0 - (double)beta1);
+    a.a2 = (float)(1.0 - (double)beta2);
+    return finish(kOptim[fmt](a));
+}
+
+int fbsr_accumulate(void* w_lp, const float* update, size_t n, int fmt, int variant, int k_bits, uint64_t seed,
+                    uint64_t offset, void* cuda_stream)
+{
+    if (bad_enum(fmt, variant, k_bits)) return FBSR_ERR_INVALID_ARG;
+    if (n > 0 && (!w_lp || !update)) return FBSR_ERR_INVALID_ARG;
+    if (misaligned(update, 4) || misaligned(w_lp, code_bytes(fmt))) return FBSR_ERR_ALIGNMENT;
+    if (n == 0) return FBSR_OK;
+    CallArgs a = base_args(OP_ACCUM, variant, k_bits, n, seed, offset, w_lp, cuda_stream);
+    a.src = update;
+    return finish(kOptim[fmt](a));
+}
+
+size_t fbsr_tile_elements(int k_bits)
+{
+    if (k_bits < 1 || k_bits > 16) return 0;
+    const int dpw = 32 / k_bits;
+    const int r0 = (dpw % 2 == 0) ? dpw / 2 : dpw;
+    const int mult = r0 >= 4 ? 1 : (4 + r0 - 1) / r0;
+    return (size_t)r0 * mult * 256;
+}
+
+size_t fbsr_round_host_min_workspace(void) { return (size_t)1 << 20; }
+
+int fbsr_round_host(const float* src_host, void* dst_host, size_t n, int fmt, int variant, int k_bits,
+                    uint64_t seed, uint64_t offset, float scale, void* dev_workspace, size_t workspace_bytes,
+                    void* cuda_stream)
+{
+    if (int rc = check_round(src_host, dst_host, n, fmt, variant, k_bits, scale)) return rc;
+    if (dev_workspace == nullptr || workspace_bytes < fbsr_round_host_min_workspace()) return FBSR_ERR_WORKSPACE;
+    if (misaligned(dev_workspace, 256)) return FBSR_ERR_ALIGNMENT;
+    if (n == 0) return FBSR_OK;
+
+    // Per-device copy stream and events, created on first use and kept for the life of the process.
+    struct Side { cudaStream_t d2h = nullptr; cudaEvent_t rounded[2] = {nullptr, nullptr}, drained[2] = {nullptr, nullptr}; bool ok = false; };
+    static Side sides[64];
+    static std::mutex mu;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return FBSR_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(mu);
+    Side& s = sides[dev];
+    if (!s.ok) {
+        if (cudaStreamCreateWithFlags(&s.d2h, cudaStreamNonBlocking) != cudaSuccess) return FBSR_ERR_CUDA;
+        for (int i = 0; i < 2; ++i) {
+            if (cudaEventCreateWithFlags(&s.rounded[i], cudaEventDisableTiming) != cudaSuccess ||
+                cudaEventCreateWithFlags(&s.drained[i], cudaEventDisableTiming) != cudaSuccess) return FBSR_ERR_CUDA;
+        }
+        s.ok = true;
+    }
+
+    const cudaStream_t main = static_cast<cudaStream_t>(cuda_stream);
+    const size_t cb = code_bytes(fmt);
+    const size_t tile = fbsr_tile_elements(k_bits);
+    // Two slots, each: chunk binary32 inputs then chunk codes, both 256-byte aligned.
+    size_t chunk = (workspace_bytes / 2 - 512) / (4 + cb);
+    chunk = chunk / tile * tile;
+    const size_t max_chunk = (size_t)1 << 26;               // keeps the first copy from delaying the first kernel
+    if (chunk > max_chunk) chunk = max_chunk / tile * tile;
+    if (chunk == 0) return FBSR_ERR_WORKSPACE;
+    char* slot_in[2]; char* slot_out[2];
+    const size_t in_bytes = (chunk * 4 + 255) / 256 * 256, out_bytes = (chunk * cb + 255) / 256 * 256;
+    for (int i = 0; i < 2; ++i) {
+        slot_in[i] = static_cast<char*>(dev_workspace) + i * (in_bytes + out_bytes);
+        slot_out[i] = slot_in[i] + in_bytes;
+    }
+    if (2 * (in_bytes + out_bytes) > workspace_bytes) return FBSR_ERR_WORKSPACE;
+
+    bool used[2] = {false, false};
+    size_t idx = 0;
+    for (size_t at = 0; at < n; at += chunk, ++idx) {
+        const int sl = (int)(idx & 1);
+        const size_t len = n - at < chunk ? n - at : chunk;
+        // the slot's previous codes must have left before its buffers are reused
+        if (used[sl] && cudaStreamWaitEvent(main, s.drained[sl], 0) != cudaSuccess) return FBSR_ERR_CUDA;
+        if (cudaMemcpyAsync(slot_in[sl], src_host + at, len * 4, cudaMemcpyHostToDevice, main) != cudaSuccess) return FBSR_ERR_CUDA;
+        CallArgs a = base_args(OP_ROUND, variant, k_bits, len, seed, offset + at, slot_out[sl], main);
+        a.src = reinterpret_cast<const float*>(slot_in[sl]); a.scale = scale;
+        if (kRound[fmt](a) != 0) return FBSR_ERR_UNSUPPORTED;
+        if (cudaEventRecord(s.rounded[sl], main) != cudaSuccess) return FBSR_ERR_CUDA;
+        if (cudaStreamWaitEvent(s.d2h, s.rounded[sl], 0) != cudaSuccess) return FBSR_ERR_CUDA;
+        if (cudaMemcpyAsync(static_cast<char*>(dst_host) + at * cb, slot_out[sl], len * cb, cudaMemcpyDeviceToHost, s.d2h) != cudaSuccess) return FBSR_ERR_CUDA;
+        if (cudaEventRecord(s.drained[sl], s.d2h) != cudaSuccess) return FBSR_ERR_CUDA;
+        used[sl] = true;
+    }
+    // join: the caller's stream finishes only after every code has reached the host
+    for (int sl = 0; sl < 2; ++sl)
+        if (used[sl] && cudaStreamWaitEvent(main, s.drained[sl], 0) != cudaSuccess) return FBSR_ERR_CUDA;
+    return cudaGetLastError() == cudaSuccess ? FBSR_OK : FBSR_ERR_CUDA;
+}
+
+uint64_t fbsr_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+const char* fbsr_status_string(int status)
+{
+    switch (status) {
+    case FBSR_OK: return "ok";
+    case FBSR_ERR_INVALID_ARG: return "invalid argument";
+    case FBSR_ERR_UNSUPPORTED: return "unsupported combination";
+    case FBSR_ERR_ALIGNMENT: return "pointer not aligned to its element size";
+    case FBSR_ERR_CUDA: return "CUDA runtime error";
+    case FBSR_ERR_WORKSPACE: return "workspace missing or too small";
+    default: return "unknown status";
+    }
+}
+
+int fbsr_version(void) { return 100; }
+
+}  // extern "C"

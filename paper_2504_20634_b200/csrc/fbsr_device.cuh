@@ -1,0 +1,193 @@
+// Device primitives for few-bit stochastic rounding on sm_100a:
+// Philox4x32-10, k-bit field extraction, the per-format integer rounder.
+//
+// Rounding of one binary32 pattern y to format (K, P, B; M), Section II-A:
+//   sh  = number of excess bits = (24 - P) + max(0, (1 - B) - exponent(y))   [Eq. (2)]
+//   m   = 24-bit integer significand of |y|, F = m >> sh = floor(sigma~)     [Eq. (3)]
+//   r   = low sh bits of m, delta~ = r / 2^sh
+// and the predicates of Section II-B / Eq. (8) become integer carries:
+//   SRFF  sigma = ((m >> (sh - N)) + n) >> N
+//   SRF   sigma = ((m >> (sh - N - 1)) + 2n + 1) >> (N + 1)
+//   SRC   sigma = (RTNE(m / 2^(sh - N)) + n) >> N
+// (a right shift by a negative amount means a left shift).  The output magnitude
+// is ((te - emin) << (P - 1)) + sigma, which carries sigma = 2^P into the exponent
+// and subnormal -> normal by the same addition [Eq. (5)].
+#pragma once
+#include <cstdint>
+#include <cuda_runtime.h>
+
+namespace fbsr {
+
+enum { BF16 = 0, FP16 = 1, E4M3 = 2, E5M2 = 3 };
+enum { SRFF = 0, SRF = 1, SRC = 2 };
+
+template <int FMT> struct Format;
+template <> struct Format<BF16> {
+    static constexpr int K = 16, P = 8, EMINB = 1;        // (1 - B) + 127: emin as a binary32 biased exponent
+    static constexpr uint32_t MAXBITS = 0x7F7F0000u;       // binary32 pattern of M
+    static constexpr uint32_t MAXCODE = 0x7F7Fu, INFCODE = 0x7F80u, NANCODE = 0x7FC0u;
+};
+template <> struct Format<FP16> {
+    static constexpr int K = 16, P = 11, EMINB = 113;
+    static constexpr uint32_t MAXBITS = 0x477FE000u;
+    static constexpr uint32_t MAXCODE = 0x7BFFu, INFCODE = 0x7C00u, NANCODE = 0x7E00u;
+};
+template <> struct Format<E4M3> {
+    static constexpr int K = 8, P = 4, EMINB = 121;
+    static constexpr uint32_t MAXBITS = 0x43E00000u;
+    static constexpr uint32_t MAXCODE = 0x7Eu, INFCODE = 0x7Eu /* no Inf: saturate */, NANCODE = 0x7Fu;
+};
+template <> struct Format<E5M2> {
+    static constexpr int K = 8, P = 3, EMINB = 113;
+    static constexpr uint32_t MAXBITS = 0x47600000u;
+    static constexpr uint32_t MAXCODE = 0x7Bu, INFCODE = 0x7Cu, NANCODE = 0x7Fu;
+};
+
+// ----------------------------------------------------------------------------
+// Philox4x32-10 (Salmon et al., SC'11).  The round keys depend only on the
+// seed: the key additions are uniform across the grid.
+// ----------------------------------------------------------------------------
+__device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
+                                               uint32_t k0, uint32_t k1)
+{
+#pragma unroll
+    for (int r = 0; r < 10; ++r) {
+        const uint64_t p0 = (uint64_t)0xD2511F53u * c0;
+        const uint64_t p1 = (uint64_t)0xCD9E8D57u * c2;
+        const uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ k0;
+        const uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ k1;
+        c1 = (uint32_t)p1;
+        c3 = (uint32_t)p0;
+        c0 = n0;
+        c2 = n2;
+        k0 += 0x9E3779B9u;
+        k1 += 0xBB67AE85u;
+    }
+    return make_uint4(c0, c1, c2, c3);
+}
+
+__device__ __forceinline__ uint4 philox_block(uint64_t block, uint32_t k0, uint32_t k1)
+{
+    return philox4x32_10((uint32_t)block, (uint32_t)(block >> 32), 0u, 0u, k0, k1);
+}
+
+// Outcome of one element for the statistics path.
+struct ElementInfo {
+    int kind;      // 0 SR-rounded, 1 NaN, 2 Inf, 3 saturated
+    int up;        // 1 if the magnitude was rounded up
+    double delta;  // delta~ = r / 2^sh, exact in binary64
+};
+
+// ----------------------------------------------------------------------------
+// One element.  ybits: the (scaled) binary32 pattern; n: the N-bit draw.
+// Returns the K-bit code.  VAR and N are ordinary arguments so that the slow
+// path can pass run-time values; the tiled kernels pass constants and the
+// branches fold away.
+// ----------------------------------------------------------------------------
+template <int FMT, bool STATS>
+__device__ __forceinline__ uint32_t round_core(uint32_t ybits, uint32_t n, const int VAR, const int N,
+                                               ElementInfo* info)
+{
+    using F = Format<FMT>;
+    constexpr int P = F::P;
+    const uint32_t mag = ybits & 0x7FFFFFFFu;
+    const uint32_t sign = (ybits >> 31) << (F::K - 1);
+    uint32_t enc;
+
+    if constexpr (FMT == BF16 && !STATS) {
+        // bfloat16 shares binary32's exponent range: sh is always 16 and the
+        // whole of Eq. (2)-(5) is one addition on the magnitude pattern.
+        uint32_t t;
+        if (VAR == SRFF || N == 16) {
+            t = mag + (n << (16 - N));
+        } else if (VAR == SRF) {
+            t = mag + (((n << 1) | 1u) << (15 - N));
+        } else {
+            const int s = 16 - N;                            // bits removed by the pre-round, >= 1
+            const uint32_t pre = (mag + ((1u << (s - 1)) - 1u) + ((mag >> s) & 1u)) & ~((1u << s) - 1u);
+            t = pre + (n << s);
+        }
+        enc = t >> 16;
+    } else {
+        const uint32_t e32 = mag >> 23;
+        const uint32_t m = (mag & 0x7FFFFFu) | (e32 ? 0x800000u : 0u);
+        const int eb = max((int)e32, 1);
+        const int te = max(eb, F::EMINB);
+        const int sh = (24 - P) + (te - eb);                 // excess bits, >= 24 - P >= 13
+        const uint32_t m6 = m << 6;                          // 6 guard positions keep every shift >= 0
+        uint32_t sig;
+        if (VAR == SRFF) {
+            const int sa = min(sh - N + 6, 31);
+            sig = ((m6 >> sa) + n) >> N;
+        } else if (VAR == SRF) {
+            const int sa = min(sh - N + 5, 31);
+            sig = ((m6 >> sa) + ((n << 1) | 1u)) >> (N + 1);
+        } else {
+            const int sa = min(sh - N + 6, 31);              // >= 3
+            const uint32_t pre = (m6 + ((1u << (sa - 1)) - 1u) + ((m6 >> sa) & 1u)) >> sa;
+            sig = (pre + n) >> N;
+        }
+        enc = ((uint32_t)(te - F::EMINB) << (P - 1)) + sig;
+        if constexpr (STATS) {
+            const uint32_t fl = m >> min(sh, 31);
+            const uint32_t r = sh < 32 ? (m & ((1u << sh) - 1u)) : m;
+            info->up = (int)(sig - fl);
+            // 2^-sh as a binary64 pattern (sh < 300 keeps it a normal double)
+            info->delta = (double)r * __longlong_as_double((long long)(1023 - sh) << 52);
+        }
+    }
+    if constexpr (STATS) info->kind = 0;
+    if (mag > F::MAXBITS) {
+        if (mag > 0x7F800000u) { enc = F::NANCODE; if constexpr (STATS) info->kind = 1; }
+        else if (mag == 0x7F800000u) { enc = F::INFCODE; if constexpr (STATS) info->kind = 2; }
+        else { enc = F::MAXCODE; if constexpr (STATS) info->kind = 3; }
+    }
+    return enc | sign;
+}
+
+// y = fl32(x * scale); a NaN input passes through so that its sign survives.
+__device__ __forceinline__ uint32_t scaled_bits(float x, float scale)
+{
+    const uint32_t xb = __float_as_uint(x);
+    if ((xb & 0x7FFFFFFFu) > 0x7F800000u) return xb;
+    return __float_as_uint(__fmul_rn(x, scale));
+}
+
+// NaNs produced by arithmetic are written as the positive quiet NaN.
+__device__ __forceinline__ uint32_t arith_bits(float y)
+{
+    const uint32_t yb = __float_as_uint(y);
+    return (yb & 0x7FFFFFFFu) > 0x7F800000u ? 0x7FC00000u : yb;
+}
+
+// Value of a stored code, Eq. (1), widened exactly to binary32.
+template <int FMT>
+__device__ __forceinline__ float decode_element(uint32_t code)
+{
+    using F = Format<FMT>;
+    constexpr int P = F::P, K = F::K;
+    if constexpr (FMT == BF16) {
+        return __uint_as_float((code & 0xFFFFu) << 16);
+    } else {
+        const uint32_t sign = ((code >> (K - 1)) & 1u) << 31;
+        const uint32_t mag = code & ((1u << (K - 1)) - 1u);
+        const uint32_t e = mag >> (P - 1), t = mag & ((1u << (P - 1)) - 1u);
+        if constexpr (FMT == E4M3) {
+            if (mag == F::NANCODE) return __uint_as_float(sign | 0x7FC00000u);
+        } else {
+            if (mag > F::INFCODE) return __uint_as_float(sign | 0x7FC00000u);
+            if (mag == F::INFCODE) return __uint_as_float(sign | 0x7F800000u);
+        }
+        uint32_t bits;
+        if (e == 0) {
+            // subnormal: t 2^(1-P) 2^(1-B), exact in binary32
+            const float v = __fmul_rn((float)t, __uint_as_float((uint32_t)(F::EMINB - (P - 1)) << 23));
+            bits = __float_as_uint(v);
+        } else {
+            bits = ((e + (uint32_t)(F::EMINB - 1)) << 23) | (t << (24 - P));
+        }
+        return __uint_as_float(sign | bits);
+    }
+}
+
+}  // namespace fbsr

@@ -1,0 +1,174 @@
+// Kernel instantiations and launch logic for one target format and one group of
+// operations.  Compiled once per (FBSR_FMT, FBSR_GROUP): FBSR_GROUP 0 = rounding
+// entry points, 1 = fused optimizer / accumulation entry points.
+#include <array>
+#include <utility>
+
+#include "fbsr_internal.h"
+#include "fbsr_kernels.cuh"
+
+#ifndef FBSR_FMT
+#error "compile with -DFBSR_FMT=0..3"
+#endif
+#ifndef FBSR_GROUP
+#error "compile with -DFBSR_GROUP=0|1"
+#endif
+
+namespace fbsr {
+namespace {
+
+constexpr int FMT = FBSR_FMT;
+constexpr int CODE_BYTES = Format<FMT>::K / 8;
+
+inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+// Host view of an Op: which pointers the tiled kernel reads with 256-bit accesses, and
+// the same Op with every pointer moved forward by h elements.
+inline bool op_aligned(const RoundOp& o, size_t h) { return aligned(o.src + h, 32); }
+inline RoundOp op_advance(RoundOp o, size_t h) { o.src += h; return o; }
+inline bool op_aligned(const SgdOp& o, size_t h) { return aligned(o.w + h, 32) && aligned(o.g + h, 32) && aligned(o.m + h, 32); }
+inline SgdOp op_advance(SgdOp o, size_t h) { o.w += h; o.g += h; o.m += h; return o; }
+inline bool op_aligned(const AdamOp& o, size_t h)
+{
+    return aligned(o.w + h, 32) && aligned(o.g + h, 32) && aligned(o.m + h, 32) && aligned(o.v + h, 32);
+}
+inline AdamOp op_advance(AdamOp o, size_t h) { o.w += h; o.g += h; o.m += h; o.v += h; return o; }
+inline bool op_aligned(const AccumOp<FMT>& o, size_t h) { return aligned(o.u + h, 32); }
+inline AccumOp<FMT> op_advance(AccumOp<FMT> o, size_t h)
+{
+    o.u += h; o.w_lp = static_cast<const char*>(o.w_lp) + h * CODE_BYTES; return o;
+}
+
+struct Plan { size_t head, n_tiles, tail_begin; };
+
+template <class Op, int VAR, int K, bool BITS>
+int launch_tiles(const Op& op, const CallArgs& a, const Plan& p)
+{
+    using T = Tile<K>;
+    auto kern = tile_kernel<Op, FMT, VAR, K, BITS>;
+    static int ctas_per_sm = 0;
+    if (ctas_per_sm == 0) {
+        int occ = 0;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kern, CTA_THREADS, 0) != cudaSuccess || occ < 1) occ = 1;
+        ctas_per_sm = occ;
+    }
+    const uint64_t want = (p.n_tiles + WARPS_PER_CTA - 1) / WARPS_PER_CTA;
+    const uint64_t cap = (uint64_t)sm_count() * ctas_per_sm;
+    const unsigned grid = (unsigned)(want < cap ? want : cap);
+    const Op adv = op_advance(op, p.head);
+    void* dst = static_cast<char*>(a.dst) + p.head * CODE_BYTES;
+    const uint64_t call0 = BITS ? 0 : (a.offset + p.head) / T::E;
+    const uint32_t* words = BITS ? a.words + p.head / T::DPW : nullptr;
+    kern<<<grid, CTA_THREADS, 0, a.stream>>>(adv, dst, p.n_tiles, call0, (uint32_t)a.seed,
+                                             (uint32_t)(a.seed >> 32), words);
+    count_launch();
+    return 0;
+}
+
+template <class Op, bool BITS, bool STATS>
+int launch_generic(const Op& op, const CallArgs& a, size_t i_begin, size_t i_end, int* n_ctas_out)
+{
+    if (n_ctas_out) *n_ctas_out = 0;
+    if (i_begin >= i_end) return 0;
+    const uint64_t E = 4u * (32u / (unsigned)a.k);
+    const uint64_t off = BITS ? 0 : a.offset;
+    const uint64_t n_calls = (off + i_end - 1) / E - (off + i_begin) / E + 1;
+    uint64_t ctas = (n_calls + CTA_THREADS - 1) / CTA_THREADS;
+    if (ctas > (uint64_t)MAX_SLOW_GRID) ctas = MAX_SLOW_GRID;
+    const uint64_t dpw = 32u / (unsigned)a.k;
+    generic_kernel<Op, FMT, BITS, STATS><<<(unsigned)ctas, CTA_THREADS, 0, a.stream>>>(
+        op, a.dst, i_begin, i_end, off, a.variant, a.k, (uint32_t)a.seed, (uint32_t)(a.seed >> 32),
+        a.words, BITS ? (a.n + dpw - 1) / dpw : 0, STATS ? a.group_size : 0, a.gsum_e, a.gsum_e2,
+        static_cast<StatsAcc*>(a.partials));
+    count_launch();
+    if (n_ctas_out) *n_ctas_out = (int)ctas;
+    return 0;
+}
+
+// Split a call into [0, head) slow, whole tiles fast, [tail_begin, n) slow.
+template <class Op, int K, bool BITS>
+Plan make_plan(const Op& op, const CallArgs& a)
+{
+    using T = Tile<K>;
+    Plan p{0, 0, 0};
+    const uint64_t off = BITS ? 0 : a.offset;
+    const size_t head = (size_t)((T::ELEMS - off % T::ELEMS) % T::ELEMS);
+    const size_t dst_align = CODE_BYTES == 2 ? 16 : 8;
+    if (head < a.n && op_aligned(op, head) &&
+        aligned(static_cast<char*>(a.dst) + head * CODE_BYTES, dst_align)) {
+        p.head = head;
+        p.n_tiles = (a.n - head) / T::ELEMS;
+    }
+    if (p.n_tiles == 0) p.head = 0;
+    p.tail_begin = p.head + p.n_tiles * T::ELEMS;
+    return p;
+}
+
+template <class Op, int VAR, int K, bool BITS>
+int run(const Op& op, const CallArgs& a)
+{
+    const Plan p = make_plan<Op, K, BITS>(op, a);
+    if (p.n_tiles == 0) return launch_generic<Op, BITS, false>(op, a, 0, a.n, nullptr);
+    launch_generic<Op, BITS, false>(op, a, 0, p.head, nullptr);
+    launch_tiles<Op, VAR, K, BITS>(op, a, p);
+    launch_generic<Op, BITS, false>(op, a, p.tail_begin, a.n, nullptr);
+    return 0;
+}
+
+// ---- (variant, k) -> instantiation
+template <class Op, bool BITS> using RunFn = int (*)(const Op&, const CallArgs&);
+
+template <class Op, bool BITS, int VAR, int... Ks>
+constexpr std::array<RunFn<Op, BITS>, 16> row_of(std::integer_sequence<int, Ks...>)
+{
+    return {{&run<Op, VAR, Ks + 1, BITS>...}};
+}
+
+template <class Op, bool BITS>
+int by_variant_and_k(const Op& op, const CallArgs& a)
+{
+    using Seq = std::make_integer_sequence<int, 16>;
+    static constexpr std::array<RunFn<Op, BITS>, 16> table[3] = {
+        row_of<Op, BITS, SRFF>(Seq{}), row_of<Op, BITS, SRF>(Seq{}), row_of<Op, BITS, SRC>(Seq{})};
+    return table[a.variant][a.k - 1](op, a);
+}
+
+}  // namespace
+
+#define FBSR_CAT_(a, b) a##b
+#define FBSR_CAT(a, b) FBSR_CAT_(a, b)
+
+#if FBSR_GROUP == 0
+int FBSR_CAT(dispatch_round_, FBSR_FMT)(const CallArgs& a)
+{
+    const RoundOp op{a.src, a.scale};
+    switch (a.op) {
+    case OP_ROUND: return by_variant_and_k<RoundOp, false>(op, a);
+    case OP_ROUND_BITS: return by_variant_and_k<RoundOp, true>(op, a);
+    case OP_ROUND_STATS: {
+        // Statistics run on the general kernel only; per-CTA partials are reduced in a fixed order.
+        int n_ctas = 0;
+        launch_generic<RoundOp, false, true>(op, a, 0, a.n, &n_ctas);
+        stats_finalize_kernel<<<1, CTA_THREADS, 0, a.stream>>>(static_cast<const StatsAcc*>(a.partials), n_ctas,
+                                                               static_cast<StatsAcc*>(a.total));
+        count_launch();
+        return 0;
+    }
+    default: return 1;
+    }
+}
+#else
+int FBSR_CAT(dispatch_optim_, FBSR_FMT)(const CallArgs& a)
+{
+    switch (a.op) {
+    case OP_SGD: return by_variant_and_k<SgdOp, false>(SgdOp{a.w, a.g, a.m, a.neg_lr, a.mu}, a);
+    case OP_ADAM:
+        return by_variant_and_k<AdamOp, false>(
+            AdamOp{a.w, a.g, a.m, a.v, a.beta1, a.beta2, a.eps, a.neg_c1, a.c2, a.a1, a.a2}, a);
+    case OP_ACCUM: return by_variant_and_k<AccumOp<FMT>, false>(AccumOp<FMT>{a.dst, a.src}, a);
+    default: return 1;
+    }
+}
+#endif
+
+}  // namespace fbsr

@@ -1,0 +1,47 @@
+// Host-side plumbing shared by the translation units of libfbsr.so (not part of the public ABI).
+#pragma once
+#include <cstddef>
+#include <cstdint>
+#include <cuda_runtime.h>
+
+namespace fbsr {
+
+enum OpKind { OP_ROUND = 0, OP_ROUND_BITS, OP_ROUND_STATS, OP_SGD, OP_ADAM, OP_ACCUM };
+
+// Everything an entry point hands to the per-format dispatcher.  Validated by the caller.
+struct CallArgs {
+    OpKind op;
+    int variant, k;
+    size_t n;
+    uint64_t seed, offset;
+    cudaStream_t stream;
+    void* dst;                      // low-precision codes (w_lp for OP_ACCUM)
+    // OP_ROUND*, OP_ACCUM (src = update)
+    const float* src;
+    float scale;
+    const uint32_t* words;          // OP_ROUND_BITS
+    // OP_ROUND_STATS
+    size_t group_size;
+    double* gsum_e;
+    double* gsum_e2;
+    void* total;                    // fbsr_stats*
+    void* partials;                 // workspace
+    // OP_SGD / OP_ADAM
+    float* w; const float* g; float* m; float* v;
+    float neg_lr, mu;                                   // SGD-momentum
+    float beta1, beta2, eps, neg_c1, c2, a1, a2;        // Adam
+};
+
+constexpr int MAX_SLOW_GRID = 148 * 8;      // CTAs of the general kernel; also the number of partial slots
+
+// One dispatcher per (format, op group); each lives in its own translation unit.
+#define FBSR_DECLARE_DISPATCH(fmt) \
+    int dispatch_round_##fmt(const CallArgs&); \
+    int dispatch_optim_##fmt(const CallArgs&);
+FBSR_DECLARE_DISPATCH(0) FBSR_DECLARE_DISPATCH(1) FBSR_DECLARE_DISPATCH(2) FBSR_DECLARE_DISPATCH(3)
+#undef FBSR_DECLARE_DISPATCH
+
+void count_launch();                         // bumps the counter behind fbsr_launch_count()
+int sm_count();                              // multiprocessors of the current device
+
+}  // namespace fbsr

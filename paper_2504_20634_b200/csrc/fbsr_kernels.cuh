@@ -1,0 +1,457 @@
+// Kernels for few-bit stochastic rounding on sm_100a.
+//
+// Two kernels serve every entry point:
+//
+//  * tile_kernel: the bandwidth path.  A warp owns a tile of ROWS rows of 256
+//    consecutive elements; in each row a lane owns 8 consecutive elements, so a
+//    warp instruction reads 1 KiB of binary32 input (one 256-bit load per lane)
+//    and writes 512 contiguous bytes of 16-bit codes (one 128-bit store per
+//    lane) or 256 bytes of 8-bit codes.  The tile size is chosen per k so that a
+//    tile is a whole number of Philox calls, evenly spread over the 32 lanes;
+//    the words go through a per-warp shared-memory buffer laid out exactly like
+//    the packed word stream of the interface, from which every lane picks the
+//    fields of its own elements.  With two draws per word a Philox call serves
+//    exactly one lane's 8 elements and the buffer is skipped.
+//
+//  * generic_kernel: any pointer alignment, any offset, heads and tails.  One
+//    thread per Philox call, scalar loads and stores, run-time k and variant,
+//    optional statistics.
+//
+// An "Op" supplies the value to be rounded: the scaled input (fbsr_round), the
+// freshly updated master weight (SGD-momentum, Adam) or the widened stored
+// weight plus its update (accumulate).
+#pragma once
+#include "fbsr_device.cuh"
+
+namespace fbsr {
+
+constexpr int WARPS_PER_CTA = 8;
+constexpr int CTA_THREADS = WARPS_PER_CTA * 32;
+constexpr int ROW_ELEMS = 256;          // 32 lanes x 8 elements
+
+template <int K> struct Tile {
+    static constexpr int DPW = 32 / K;                        // draws per word
+    static constexpr int E = 4 * DPW;                         // elements per Philox call
+    static constexpr int R0 = (DPW % 2 == 0) ? DPW / 2 : DPW; // rows holding 32 (or 64) whole calls
+    static constexpr int MULT = R0 >= 4 ? 1 : (4 + R0 - 1) / R0;
+    static constexpr int ROWS = R0 * MULT;
+    static constexpr int ELEMS = ROWS * ROW_ELEMS;
+    static constexpr int CALLS = ELEMS / E;                   // Philox calls per tile
+    static constexpr int WORDS = ELEMS / DPW;                 // random words per tile
+    static constexpr uint32_t MASK = (1u << K) - 1u;
+    static_assert(ELEMS % E == 0 && CALLS % 32 == 0, "tile must hold whole calls, evenly per lane");
+};
+
+// ---------------------------------------------------------------------------- vector memory access
+struct F8 { float4 a, b; };
+
+__device__ __forceinline__ F8 load_f8_stream(const float* p)
+{
+    // 256-bit read-only load that does not allocate in L1: the data is used once.
+    F8 v;
+    asm volatile("ld.global.nc.L1::no_allocate.L2::evict_first.v8.f32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=f"(v.a.x), "=f"(v.a.y), "=f"(v.a.z), "=f"(v.a.w),
+                   "=f"(v.b.x), "=f"(v.b.y), "=f"(v.b.z), "=f"(v.b.w)
+                 : "l"(p));
+    return v;
+}
+
+__device__ __forceinline__ F8 load_f8(const float* p)
+{
+    F8 v;
+    asm volatile("ld.global.v8.f32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=f"(v.a.x), "=f"(v.a.y), "=f"(v.a.z), "=f"(v.a.w),
+                   "=f"(v.b.x), "=f"(v.b.y), "=f"(v.b.z), "=f"(v.b.w)
+                 : "l"(p));
+    return v;
+}
+
+__device__ __forceinline__ void store_f8(float* p, const float (&y)[8])
+{
+    asm volatile("st.global.v8.f32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
+                 :: "l"(p), "f"(y[0]), "f"(y[1]), "f"(y[2]), "f"(y[3]),
+                    "f"(y[4]), "f"(y[5]), "f"(y[6]), "f"(y[7]) : "memory");
+}
+
+__device__ __forceinline__ void unpack(const F8& v, float (&x)[8])
+{
+    x[0] = v.a.x; x[1] = v.a.y; x[2] = v.a.z; x[3] = v.a.w;
+    x[4] = v.b.x; x[5] = v.b.y; x[6] = v.b.z; x[7] = v.b.w;
+}
+
+template <int FMT>
+__device__ __forceinline__ void store_codes8(void* dst, size_t elem, const uint32_t (&c)[8])
+{
+    if constexpr (Format<FMT>::K == 16) {
+        uint4 v;
+        v.x = c[0] | (c[1] << 16); v.y = c[2] | (c[3] << 16);
+        v.z = c[4] | (c[5] << 16); v.w = c[6] | (c[7] << 16);
+        __stcs(reinterpret_cast<uint4*>(static_cast<uint16_t*>(dst) + elem), v);
+    } else {
+        uint2 v;
+        v.x = c[0] | (c[1] << 8) | (c[2] << 16) | (c[3] << 24);
+        v.y = c[4] | (c[5] << 8) | (c[6] << 16) | (c[7] << 24);
+        __stcs(reinterpret_cast<uint2*>(static_cast<uint8_t*>(dst) + elem), v);
+    }
+}
+
+template <int FMT>
+__device__ __forceinline__ void store_code1(void* dst, size_t elem, uint32_t c)
+{
+    if constexpr (Format<FMT>::K == 16) static_cast<uint16_t*>(dst)[elem] = (uint16_t)c;
+    else static_cast<uint8_t*>(dst)[elem] = (uint8_t)c;
+}
+
+// ---------------------------------------------------------------------------- Ops
+// fetch(): issue the loads of 8 consecutive elements; finish(): produce the 8
+// patterns to round (and write back whatever state the op updates);
+// scalar(): the same for one element on the slow path.
+
+struct RoundOp {
+    const float* src;
+    float scale;
+    struct Regs { F8 x; };
+    __device__ __forceinline__ void fetch(size_t elem, Regs& r) const { r.x = load_f8_stream(src + elem); }
+    __device__ __forceinline__ void finish(size_t, const Regs& r, uint32_t (&y)[8]) const
+    {
+        float x[8];
+        unpack(r.x, x);
+#pragma unroll
+        for (int c = 0; c < 8; ++c) y[c] = scaled_bits(x[c], scale);
+    }
+    __device__ __forceinline__ uint32_t scalar(size_t i) const { return scaled_bits(src[i], scale); }
+};
+
+// m' = fma(mu, m, g);  w' = fma(-lr, m', w)
+struct SgdOp {
+    float* w; const float* g; float* m;
+    float neg_lr, mu;
+    struct Regs { F8 w, g, m; };
+    __device__ __forceinline__ void step(float& wv, float gv, float& mv) const
+    {
+        mv = __fmaf_rn(mu, mv, gv);
+        wv = __fmaf_rn(neg_lr, mv, wv);
+    }
+    __device__ __forceinline__ void fetch(size_t elem, Regs& r) const
+    {
+        r.w = load_f8(w + elem); r.g = load_f8_stream(g + elem); r.m = load_f8(m + elem);
+    }
+    __device__ __forceinline__ void finish(size_t elem, const Regs& r, uint32_t (&y)[8]) const
+    {
+        float wv[8], gv[8], mv[8];
+        unpack(r.w, wv); unpack(r.g, gv); unpack(r.m, mv);
+#pragma unroll
+        for (int c = 0; c < 8; ++c) { step(wv[c], gv[c], mv[c]); y[c] = arith_bits(wv[c]); }
+        store_f8(w + elem, wv); store_f8(m + elem, mv);
+    }
+    __device__ __forceinline__ uint32_t scalar(size_t i) const
+    {
+        float wv = w[i], mv = m[i];
+        step(wv, g[i], mv);
+        w[i] = wv; m[i] = mv;
+        return arith_bits(wv);
+    }
+};
+
+// m' = fma(b1, m, a1 g); v' = fma(b2, v, (a2 g) g); d = sqrt(v') c2 + eps; w' = fma(-c1, m'/d, w)
+struct AdamOp {
+    float* w; const float* g; float* m; float* v;
+    float beta1, beta2, eps, neg_c1, c2, a1, a2;
+    struct Regs { F8 w, g, m, v; };
+    __device__ __forceinline__ void step(float& wv, float gv, float& mv, float& vv) const
+    {
+        mv = __fmaf_rn(beta1, mv, __fmul_rn(a1, gv));
+        vv = __fmaf_rn(beta2, vv, __fmul_rn(__fmul_rn(a2, gv), gv));
+        const float d = __fadd_rn(__fmul_rn(__fsqrt_rn(vv), c2), eps);
+        wv = __fmaf_rn(neg_c1, __fdiv_rn(mv, d), wv);
+    }
+    __device__ __forceinline__ void fetch(size_t elem, Regs& r) const
+    {
+        r.w = load_f8(w + elem); r.g = load_f8_stream(g + elem);
+        r.m = load_f8(m + elem); r.v = load_f8(v + elem);
+    }
+    __device__ __forceinline__ void finish(size_t elem, const Regs& r, uint32_t (&y)[8]) const
+    {
+        float wv[8], gv[8], mv[8], vv[8];
+        unpack(r.w, wv); unpack(r.g, gv); unpack(r.m, mv); unpack(r.v, vv);
+#pragma unroll
+        for (int c = 0; c < 8; ++c) { step(wv[c], gv[c], mv[c], vv[c]); y[c] = arith_bits(wv[c]); }
+        store_f8(w + elem, wv); store_f8(m + elem, mv); store_f8(v + elem, vv);
+    }
+    __device__ __forceinline__ uint32_t scalar(size_t i) const
+    {
+        float wv = w[i], mv = m[i], vv = v[i];
+        step(wv, g[i], mv, vv);
+        w[i] = wv; m[i] = mv; v[i] = vv;
+        return arith_bits(wv);
+    }
+};
+
+// y = fl32(value(w_lp) + u); the codes are rewritten in place by the caller of finish()
+template <int FMT>
+struct AccumOp {
+    const void* w_lp; const float* u;
+    struct Regs { F8 u; uint4 c; };
+    __device__ __forceinline__ void fetch(size_t elem, Regs& r) const
+    {
+        r.u = load_f8_stream(u + elem);
+        if constexpr (Format<FMT>::K == 16) {
+            r.c = *reinterpret_cast<const uint4*>(static_cast<const uint16_t*>(w_lp) + elem);
+        } else {
+            const uint2 t = *reinterpret_cast<const uint2*>(static_cast<const uint8_t*>(w_lp) + elem);
+            r.c = make_uint4(t.x, t.y, 0u, 0u);
+        }
+    }
+    __device__ __forceinline__ void finish(size_t, const Regs& r, uint32_t (&y)[8]) const
+    {
+        float uv[8];
+        unpack(r.u, uv);
+        const uint32_t cw[4] = {r.c.x, r.c.y, r.c.z, r.c.w};
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+            uint32_t code;
+            if constexpr (Format<FMT>::K == 16) code = (cw[c >> 1] >> ((c & 1) * 16)) & 0xFFFFu;
+            else code = (cw[c >> 2] >> ((c & 3) * 8)) & 0xFFu;
+            y[c] = arith_bits(__fadd_rn(decode_element<FMT>(code), uv[c]));
+        }
+    }
+    __device__ __forceinline__ uint32_t scalar(size_t i) const
+    {
+        uint32_t code;
+        if constexpr (Format<FMT>::K == 16) code = static_cast<const uint16_t*>(w_lp)[i];
+        else code = static_cast<const uint8_t*>(w_lp)[i];
+        return arith_bits(__fadd_rn(decode_element<FMT>(code), u[i]));
+    }
+};
+
+// ---------------------------------------------------------------------------- draws from a word buffer
+// wb: the tile's packed word stream; p0: tile-relative index of the lane's first element (multiple of 8).
+template <int K>
+__device__ __forceinline__ void draws8(const uint32_t* wb, int p0, uint32_t (&n)[8])
+{
+    using T = Tile<K>;
+    constexpr int DPW = T::DPW;
+    if constexpr (DPW >= 8 && (DPW & (DPW - 1)) == 0) {
+        const uint32_t w = wb[p0 / DPW] >> ((p0 % DPW) * K);          // all 8 fields sit in one word
+#pragma unroll
+        for (int c = 0; c < 8; ++c) n[c] = (w >> (c * K)) & T::MASK;
+    } else if constexpr (DPW == 4) {
+        const uint2 w = *reinterpret_cast<const uint2*>(wb + p0 / 4);
+#pragma unroll
+        for (int c = 0; c < 8; ++c) n[c] = ((c < 4 ? w.x : w.y) >> ((c & 3) * K)) & T::MASK;
+    } else if constexpr (DPW == 2) {
+        const uint4 w = *reinterpret_cast<const uint4*>(wb + p0 / 2);
+        const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+        for (int c = 0; c < 8; ++c) n[c] = (ww[c >> 1] >> ((c & 1) * K)) & T::MASK;
+    } else {
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+            const int p = p0 + c, q = p / DPW, f = p - q * DPW;
+            n[c] = (wb[q] >> (f * K)) & T::MASK;
+        }
+    }
+}
+
+template <int K>
+__device__ __forceinline__ void draws8_from_call(const uint4& w, uint32_t (&n)[8])
+{
+    static_assert(Tile<K>::DPW == 2, "one Philox call per 8 elements only with two draws per word");
+    const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+    for (int c = 0; c < 8; ++c) n[c] = (ww[c >> 1] >> ((c & 1) * K)) & Tile<K>::MASK;
+}
+
+// ---------------------------------------------------------------------------- the bandwidth kernel
+// Elements [0, n_tiles * ELEMS) relative to the pointers held by op/dst.
+// call0: global index of the Philox call that serves element 0 (Philox source), or
+// words: the packed word stream whose word 0 serves element 0 (supplied bits).
+template <class Op, int FMT, int VAR, int K, bool BITS>
+__global__ void __launch_bounds__(CTA_THREADS)
+tile_kernel(const Op op, void* __restrict__ dst, const uint64_t n_tiles, const uint64_t call0,
+            const uint32_t k0, const uint32_t k1, const uint32_t* __restrict__ words)
+{
+    using T = Tile<K>;
+    constexpr bool OWN_CALL = (T::DPW == 2) && !BITS;      // a call serves exactly one lane-row
+    __shared__ __align__(16) uint32_t wordbuf[WARPS_PER_CTA][OWN_CALL ? 4 : T::WORDS];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    uint32_t* wb = wordbuf[warp];
+
+    for (uint64_t tile = (uint64_t)blockIdx.x * WARPS_PER_CTA + warp; tile < n_tiles;
+         tile += (uint64_t)gridDim.x * WARPS_PER_CTA) {
+        const size_t e0 = (size_t)tile * T::ELEMS;
+        const uint64_t tile_call0 = call0 + tile * T::CALLS;
+
+        if constexpr (BITS) {
+            const uint32_t* src_words = words + tile * T::WORDS;
+#pragma unroll
+            for (int j = 0; j < T::WORDS / 32; ++j) wb[j * 32 + lane] = __ldg(src_words + j * 32 + lane);
+            __syncwarp();
+        } else if constexpr (!OWN_CALL) {
+#pragma unroll
+            for (int j = 0; j < T::CALLS / 32; ++j) {
+                const int c = j * 32 + lane;
+                *reinterpret_cast<uint4*>(wb + 4 * c) = philox_block(tile_call0 + c, k0, k1);
+            }
+            __syncwarp();
+        }
+
+#pragma unroll
+        for (int rb = 0; rb < T::ROWS; rb += 4) {
+            typename Op::Regs regs[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                if (rb + j < T::ROWS) op.fetch(e0 + (rb + j) * ROW_ELEMS + lane * 8, regs[j]);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                if (rb + j < T::ROWS) {
+                    const int p0 = (rb + j) * ROW_ELEMS + lane * 8;
+                    uint32_t y[8], n[8], c[8];
+                    op.finish(e0 + p0, regs[j], y);
+                    if constexpr (OWN_CALL) {
+                        const uint4 w = philox_block(tile_call0 + (rb + j) * 32 + lane, k0, k1);
+                        draws8_from_call<K>(w, n);
+                    } else {
+                        draws8<K>(wb, p0, n);
+                    }
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) c[i] = round_core<FMT, false>(y[i], n[i], VAR, K, nullptr);
+                    store_codes8<FMT>(dst, e0 + p0, c);
+                }
+            }
+        }
+        if constexpr (!OWN_CALL) __syncwarp();      // the buffer is rewritten by the next tile
+    }
+}
+
+// ---------------------------------------------------------------------------- statistics
+struct StatsAcc {
+    unsigned long long n_finite, n_up, n_nan, n_inf, n_sat;
+    double sum_e, sum_e2, sum_signed_e, sum_abs_e;
+};
+
+__device__ __forceinline__ void stats_zero(StatsAcc& a)
+{
+    a.n_finite = a.n_up = a.n_nan = a.n_inf = a.n_sat = 0ull;
+    a.sum_e = a.sum_e2 = a.sum_signed_e = a.sum_abs_e = 0.0;
+}
+
+__device__ __forceinline__ void stats_add(StatsAcc& a, const StatsAcc& b)
+{
+    a.n_finite += b.n_finite; a.n_up += b.n_up; a.n_nan += b.n_nan; a.n_inf += b.n_inf; a.n_sat += b.n_sat;
+    a.sum_e += b.sum_e; a.sum_e2 += b.sum_e2; a.sum_signed_e += b.sum_signed_e; a.sum_abs_e += b.sum_abs_e;
+}
+
+__device__ __forceinline__ StatsAcc stats_shfl_down(const StatsAcc& a, int d)
+{
+    StatsAcc b;
+    b.n_finite = __shfl_down_sync(0xFFFFFFFFu, a.n_finite, d);
+    b.n_up = __shfl_down_sync(0xFFFFFFFFu, a.n_up, d);
+    b.n_nan = __shfl_down_sync(0xFFFFFFFFu, a.n_nan, d);
+    b.n_inf = __shfl_down_sync(0xFFFFFFFFu, a.n_inf, d);
+    b.n_sat = __shfl_down_sync(0xFFFFFFFFu, a.n_sat, d);
+    b.sum_e = __shfl_down_sync(0xFFFFFFFFu, a.sum_e, d);
+    b.sum_e2 = __shfl_down_sync(0xFFFFFFFFu, a.sum_e2, d);
+    b.sum_signed_e = __shfl_down_sync(0xFFFFFFFFu, a.sum_signed_e, d);
+    b.sum_abs_e = __shfl_down_sync(0xFFFFFFFFu, a.sum_abs_e, d);
+    return b;
+}
+
+// Fixed-order reduction over the CTA; the result is valid in thread 0.
+__device__ __forceinline__ void stats_cta_reduce(StatsAcc& a)
+{
+    __shared__ StatsAcc per_warp[WARPS_PER_CTA];
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) stats_add(a, stats_shfl_down(a, d));
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (lane == 0) per_warp[warp] = a;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        for (int w = 1; w < WARPS_PER_CTA; ++w) stats_add(a, per_warp[w]);
+    }
+}
+
+// ---------------------------------------------------------------------------- the slow, general kernel
+// Elements [i_begin, i_end) of the call.  One thread per Philox call (or per group of four supplied words).
+template <class Op, int FMT, bool BITS, bool STATS>
+__global__ void __launch_bounds__(CTA_THREADS)
+generic_kernel(const Op op, void* __restrict__ dst, const uint64_t i_begin, const uint64_t i_end,
+               const uint64_t offset, const int variant, const int k, const uint32_t k0, const uint32_t k1,
+               const uint32_t* __restrict__ words, const uint64_t n_words,
+               const uint64_t group_size, double* __restrict__ gsum_e, double* __restrict__ gsum_e2,
+               StatsAcc* __restrict__ partials)
+{
+    const uint32_t dpw = 32u / (uint32_t)k, E = 4u * dpw, mask = (1u << k) - 1u;
+    const uint64_t g_first = offset + i_begin, g_last = offset + i_end;     // [g_first, g_last)
+    const uint64_t call_first = g_first / E;
+    const uint64_t n_calls = g_first < g_last ? (g_last - 1) / E - call_first + 1 : 0;
+    StatsAcc acc;
+    if constexpr (STATS) stats_zero(acc);
+
+    for (uint64_t b = (uint64_t)blockIdx.x * CTA_THREADS + threadIdx.x; b < n_calls;
+         b += (uint64_t)gridDim.x * CTA_THREADS) {
+        const uint64_t call = call_first + b;
+        const uint64_t g_lo = max(call * E, g_first), g_hi = min((call + 1) * E, g_last);
+        uint32_t w[4];
+        if constexpr (BITS) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) w[j] = call * 4 + j < n_words ? words[call * 4 + j] : 0u;
+        } else {
+            const uint4 o = philox_block(call, k0, k1);
+            w[0] = o.x; w[1] = o.y; w[2] = o.z; w[3] = o.w;
+        }
+        uint64_t cur_group = ~0ull;
+        double ge = 0.0, ge2 = 0.0;
+        for (uint64_t g = g_lo; g < g_hi; ++g) {
+            const uint64_t i = g - offset;
+            const uint32_t j = (uint32_t)(g - call * E);
+            const uint32_t ws = j / dpw, f = j - ws * dpw;
+            const uint32_t word = ws == 0 ? w[0] : ws == 1 ? w[1] : ws == 2 ? w[2] : w[3];
+            const uint32_t n = (word >> (f * k)) & mask;
+            const uint32_t y = op.scalar(i);
+            ElementInfo info;
+            const uint32_t code = round_core<FMT, STATS>(y, n, variant, k, &info);
+            store_code1<FMT>(dst, i, code);
+            if constexpr (STATS) {
+                if (info.kind == 0) {
+                    const double e = (double)info.up - info.delta;
+                    const double e2 = e * e;
+                    acc.n_finite += 1; acc.n_up += (unsigned)info.up;
+                    acc.sum_e += e; acc.sum_e2 += e2;
+                    acc.sum_signed_e += (y >> 31) ? -e : e;
+                    acc.sum_abs_e += fabs(e);
+                    if (group_size) {
+                        const uint64_t grp = i / group_size;
+                        if (grp != cur_group) {
+                            if (cur_group != ~0ull) { atomicAdd(gsum_e + cur_group, ge); atomicAdd(gsum_e2 + cur_group, ge2); }
+                            cur_group = grp; ge = 0.0; ge2 = 0.0;
+                        }
+                        ge += e; ge2 += e2;
+                    }
+                } else if (info.kind == 1) acc.n_nan += 1;
+                else if (info.kind == 2) acc.n_inf += 1;
+                else acc.n_sat += 1;
+            }
+        }
+        if constexpr (STATS) {
+            if (cur_group != ~0ull) { atomicAdd(gsum_e + cur_group, ge); atomicAdd(gsum_e2 + cur_group, ge2); }
+        }
+    }
+    if constexpr (STATS) {
+        stats_cta_reduce(acc);
+        if (threadIdx.x == 0) partials[blockIdx.x] = acc;
+    }
+}
+
+// Sum the per-CTA partials in a fixed order into the caller's fbsr_stats (same layout as StatsAcc).
+static __global__ void __launch_bounds__(CTA_THREADS)
+stats_finalize_kernel(const StatsAcc* __restrict__ partials, const int n_partials, StatsAcc* __restrict__ total)
+{
+    StatsAcc acc;
+    stats_zero(acc);
+    for (int i = threadIdx.x; i < n_partials; i += CTA_THREADS) stats_add(acc, partials[i]);
+    stats_cta_reduce(acc);
+    if (threadIdx.x == 0) *total = acc;
+}
+
+}  // namespace fbsr
