@@ -1,0 +1,76 @@
+"""One small, self-contained invocation of a single kernel, for profilers and quick timing.
+
+    python -m paper_2504_20634_b200.profile_case --op round --fmt bf16 --variant srf --k 4 --log2n 26 --iters 5
+
+Inputs are the synthetic 'bandwidth sweep' distribution (seed 1234).  Prints the mean
+CUDA-event time per launch and the algorithmic bandwidth.  With --log2n 26 the case holds
+well under 1 GiB on the device and still exceeds the L2 capacity.
+"""
+import argparse
+import json
+
+import torch
+
+import paper_2504_20634_b200 as fbsr
+from paper_2504_20634_b200 import workloads
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--op", default="round", choices=["round", "sgd", "adam", "accumulate", "stats", "bits"])
+    ap.add_argument("--fmt", default="bf16")
+    ap.add_argument("--variant", default="srf")
+    ap.add_argument("--k", type=int, default=4)
+    ap.add_argument("--log2n", type=int, default=26)
+    ap.add_argument("--iters", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=2)
+    args = ap.parse_args()
+
+    n = 1 << args.log2n
+    dev = torch.device("cuda", 0)
+    x = workloads.bandwidth_sweep(n, seed=1234, device=dev)
+    code_bytes = 2 if args.fmt in ("bf16", "fp16") else 1
+    out = torch.empty(n, dtype=fbsr.CODE_DTYPE[args.fmt], device=dev)
+    if args.op == "round":
+        bytes_per_elem = 4 + code_bytes
+        run = lambda s: fbsr.fbsr_round(x, args.fmt, args.variant, args.k, seed=1234, out=out)
+    elif args.op == "bits":
+        dpw = 32 // args.k
+        words = torch.randint(0, 2 ** 31, ((n + dpw - 1) // dpw,), device=dev, dtype=torch.int32).view(torch.uint32)
+        bytes_per_elem = 4 + code_bytes + 4.0 / dpw
+        run = lambda s: fbsr.fbsr_round_bits(x, args.fmt, args.variant, args.k, words, out=out)
+    elif args.op == "stats":
+        bytes_per_elem = 4 + code_bytes
+        run = lambda s: fbsr.fbsr_round_stats(x, args.fmt, args.variant, args.k, seed=1234, out=out)
+    elif args.op == "accumulate":
+        x.mul_(1e-3)
+        out.copy_(workloads.accumulation_weights(n, device=dev) if args.fmt == "bf16" else torch.zeros_like(out))
+        bytes_per_elem = 4 + 2 * code_bytes
+        run = lambda s: fbsr.fbsr_accumulate(out, x, args.fmt, args.variant, args.k, seed=s)
+    else:
+        w, m, v = workloads.optimizer_state(n, device=dev)
+        g = workloads.optimizer_grad(n, 1, device=dev)
+        if args.op == "sgd":
+            bytes_per_elem = 20 + code_bytes
+            run = lambda s: fbsr.fbsr_sgd_update(w, g, m, args.fmt, args.variant, args.k, s, 0, 1e-4, 0.9, out=out)
+        else:
+            bytes_per_elem = 28 + code_bytes
+            run = lambda s: fbsr.fbsr_adam_update(w, g, m, v, args.fmt, args.variant, args.k, s, 0, 1e-4, 0.9, 0.999,
+                                                  1e-8, s, out=out)
+    for s in range(1, args.warmup + 1):
+        run(s)
+    torch.cuda.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for s in range(args.iters):
+        run(args.warmup + 1 + s)
+    b.record()
+    torch.cuda.synchronize()
+    ms = a.elapsed_time(b) / args.iters
+    print(json.dumps({"op": args.op, "fmt": args.fmt, "variant": args.variant, "k": args.k, "n": n,
+                      "ms_per_launch": ms, "GB/s": bytes_per_elem * n / (ms * 1e-3) / 1e9,
+                      "Gelem/s": n / (ms * 1e-3) / 1e9}))
+
+
+if __name__ == "__main__":
+    main()
