@@ -54,7 +54,8 @@ typedef enum {
     FBSR_ERR_UNSUPPORTED = 2, /* a combination this build does not implement */
     FBSR_ERR_ALIGNMENT = 3,   /* a pointer is not aligned to its element size */
     FBSR_ERR_CUDA = 4,        /* the CUDA runtime reported an error at launch */
-    FBSR_ERR_WORKSPACE = 5    /* workspace missing or too small */
+    FBSR_ERR_WORKSPACE = 5,   /* workspace missing or too small */
+    FBSR_ERR_TOO_LARGE = 6    /* n exceeds the limit of an entry point with built-in scratch */
 } fbsr_status;
 
 /* Target formats (K, P, B; M), Section II.  P counts the hidden bit. */
@@ -120,6 +121,41 @@ int fbsr_round_stats(const float* src, void* dst, size_t n, int fmt, int variant
                      uint64_t seed, uint64_t offset, float scale, size_t group_size,
                      double* group_sum_e, double* group_sum_e2, fbsr_stats* total,
                      void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* fbsr_round_stats_noalloc -- fbsr_round_stats without a workspace argument.
+ * (The paper has no counterpart; this exists for the sake of callers, see below.)
+ *
+ * Who it is for: code that may not allocate device memory at the point where it
+ * wants rounding statistics -- a step that runs inside a memory pool whose size was
+ * fixed at start-up, a plugin inside someone else's process that must not touch
+ * the allocator, a monitoring hook on a device that is already full.  Such a
+ * caller cannot provide the scratch that fbsr_round_stats needs for its per-CTA
+ * partial sums, so this variant keeps that scratch inside the library: a
+ * file-scope device array of FBSR_NOALLOC_SCRATCH_BYTES (85,248 bytes), which
+ * every GPU that loads libfbsr.so holds until the process exits.  The call itself
+ * performs no cudaMalloc / cudaFree and calls no allocating routine.
+ *
+ * Arguments and results are those of fbsr_round_stats (same kernels, same fixed
+ * reduction order, so totals are bit-identical to it); src, dst, the group arrays
+ * and `total` are still the caller's.
+ *   - n must not exceed FBSR_NOALLOC_MAX_ELEMENTS (2^31); larger calls return
+ *     FBSR_ERR_TOO_LARGE and do nothing.  The limit bounds how long one call can
+ *     occupy the shared scratch.
+ *   - The first call on each device looks up the device address of the scratch
+ *     array (cudaGetSymbolAddress) with that device current; make that first
+ *     call outside any stream capture.
+ *   - All calls on a device share the one array.  It keeps whatever the previous
+ *     call left there; nothing in it has to start at zero, because every slot a
+ *     call reads is first written by that same call.  Two calls that can overlap
+ *     on the GPU (different streams without an ordering between them) race on
+ *     it and give undefined statistics: order them, or use fbsr_round_stats with
+ *     separate workspaces. */
+#define FBSR_NOALLOC_SCRATCH_BYTES 85248u
+#define FBSR_NOALLOC_MAX_ELEMENTS ((size_t)1 << 31)
+int fbsr_round_stats_noalloc(const float* src, void* dst, size_t n, int fmt, int variant, int k_bits,
+                             uint64_t seed, uint64_t offset, float scale, size_t group_size,
+                             double* group_sum_e, double* group_sum_e2, fbsr_stats* total,
+                             void* cuda_stream);
 
 /* fbsr_sgd_update -- last line of Algorithm 1 with a binary32 master copy:
  *     m' = fma(mu, m, g);  w' = fma(-lr, m', w);  dst = FBSR(w')

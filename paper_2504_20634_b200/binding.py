@@ -43,6 +43,8 @@ def _load():
     L.fbsr_stats_workspace_bytes.argtypes = []
     L.fbsr_stats_workspace_bytes.restype = sz
     L.fbsr_round_stats.argtypes = [vp, vp, sz, i, i, i, u64, u64, f, sz, vp, vp, vp, vp, sz, vp]
+    L.fbsr_round_stats_noalloc.argtypes = [vp, vp, sz, i, i, i, u64, u64, f, sz, vp, vp, vp, vp]
+    L.fbsr_round_stats_noalloc.restype = i
     L.fbsr_sgd_update.argtypes = [vp, vp, vp, vp, sz, i, i, i, u64, u64, f, f, vp]
     L.fbsr_adam_update.argtypes = [vp, vp, vp, vp, vp, sz, i, i, i, u64, u64, f, f, f, f, i, vp]
     L.fbsr_accumulate.argtypes = [vp, vp, sz, i, i, i, u64, u64, vp]
@@ -167,6 +169,28 @@ def fbsr_round_stats(src, fmt, variant, k_bits, seed, offset=0, scale=1.0, group
                "fbsr_round_stats")
     st = FbsrStats.from_buffer_copy(total.cpu().numpy().tobytes())
     return out, {name: getattr(st, name) for name, _ in FbsrStats._fields_}, ge[:groups], ge2[:groups]
+
+
+def fbsr_round_stats_noalloc(src, out, total, fmt, variant, k_bits, seed, offset=0, scale=1.0, group_size=0,
+                             group_sum_e=None, group_sum_e2=None):
+    """fbsr_round_stats for callers that cannot allocate: every buffer (codes `out`, the 72-byte
+    `total`, the optional group arrays) is supplied by the caller and the library's own built-in
+    scratch is used, so neither this wrapper nor the C call allocates anything.  Returns None;
+    read `total` (uint8[72], layout of FbsrStats) after synchronising the stream."""
+    pe = ctypes.c_void_p(group_sum_e.data_ptr()) if group_sum_e is not None else None
+    pe2 = ctypes.c_void_p(group_sum_e2.data_ptr()) if group_sum_e2 is not None else None
+    with torch.cuda.device(src.device):
+        _check(_L.fbsr_round_stats_noalloc(_dev(src, torch.float32, "src"),
+                                           _dev(out, CODE_DTYPE[_fmt_name(fmt)], "out"), src.numel(), _fmt(fmt),
+                                           _var(variant), k_bits, seed, offset, scale, group_size, pe, pe2,
+                                           _dev(total, torch.uint8, "total"), _stream(src)),
+               "fbsr_round_stats_noalloc")
+
+
+def stats_from_bytes(total):
+    """Decode a 72-byte device or host uint8 tensor holding an fbsr_stats record."""
+    st = FbsrStats.from_buffer_copy(total.cpu().numpy().tobytes())
+    return {name: getattr(st, name) for name, _ in FbsrStats._fields_}
 
 
 def fbsr_sgd_update(master_w, grad, momentum, fmt, variant, k_bits, seed, offset, lr, mu, out=None):

@@ -111,6 +111,48 @@ int fbsr_round_stats(const float* src, void* dst, size_t n, int fmt, int variant
     return finish(kRound[fmt](a));
 }
 
+}  // extern "C"
+
+// Scratch of the no-allocation statistics entry point: one slot per CTA of the general kernel.
+// In host code this name is only a handle for cudaGetSymbolAddress, never a device address.
+static __device__ __align__(256) unsigned char g_noalloc_stats_scratch[FBSR_NOALLOC_SCRATCH_BYTES];
+static_assert(FBSR_NOALLOC_SCRATCH_BYTES == MAX_SLOW_GRID * sizeof(fbsr_stats), "scratch must hold one partial per CTA");
+
+// Device address of the scratch array on the current device, looked up once per device.
+static int noalloc_scratch_address(void** out)
+{
+    static void* addr[64] = {nullptr};
+    static std::mutex mu;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return FBSR_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(mu);
+    if (addr[dev] == nullptr) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_noalloc_stats_scratch) != cudaSuccess || p == nullptr) {
+            cudaGetLastError();
+            return FBSR_ERR_CUDA;
+        }
+        addr[dev] = p;
+    }
+    *out = addr[dev];
+    return FBSR_OK;
+}
+
+extern "C" {
+
+int fbsr_round_stats_noalloc(const float* src, void* dst, size_t n, int fmt, int variant, int k_bits, uint64_t seed,
+                             uint64_t offset, float scale, size_t group_size, double* group_sum_e,
+                             double* group_sum_e2, fbsr_stats* total, void* cuda_stream)
+{
+    if (n > FBSR_NOALLOC_MAX_ELEMENTS) return FBSR_ERR_TOO_LARGE;
+    void* scratch = nullptr;
+    if (int rc = noalloc_scratch_address(&scratch)) return rc;
+    // Every partial slot that the final reduction reads is written by this call's own CTAs first,
+    // so the array needs no clearing between calls.
+    return fbsr_round_stats(src, dst, n, fmt, variant, k_bits, seed, offset, scale, group_size, group_sum_e,
+                            group_sum_e2, total, scratch, FBSR_NOALLOC_SCRATCH_BYTES, cuda_stream);
+}
+
 int fbsr_sgd_update(float* master_w, const float* grad, float* momentum, void* dst_lp, size_t n, int fmt,
                     int variant, int k_bits, uint64_t seed, uint64_t offset, float lr, float mu, void* cuda_stream)
 {
@@ -246,6 +288,7 @@ const char* fbsr_status_string(int status)
     case FBSR_ERR_ALIGNMENT: return "pointer not aligned to its element size";
     case FBSR_ERR_CUDA: return "CUDA runtime error";
     case FBSR_ERR_WORKSPACE: return "workspace missing or too small";
+    case FBSR_ERR_TOO_LARGE: return "n exceeds the limit of this entry point's built-in scratch";
     default: return "unknown status";
     }
 }
