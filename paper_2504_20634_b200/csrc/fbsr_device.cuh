@@ -145,6 +145,122 @@ __device__ __forceinline__ uint32_t round_core(uint32_t ybits, uint32_t n, const
     return enc | sign;
 }
 
+// ----------------------------------------------------------------------------
+// Eight draws of one lane, normalised: element c's field starts at bit
+// (c % G) * K of word u[c / G].  The field is never isolated on its own; it is
+// shifted straight to where the rounder adds it (two integer instructions).
+// ----------------------------------------------------------------------------
+template <int K> struct Draws8 {
+    static constexpr int DPW = 32 / K;
+    static constexpr bool POW2 = (DPW & (DPW - 1)) == 0;
+    static constexpr int G = POW2 ? (DPW >= 8 ? 8 : DPW) : (4 * K <= 32 ? 4 : 2);
+    static constexpr uint32_t MASK = (1u << K) - 1u;
+    uint32_t u[8 / G];
+
+    // Field of element c moved so that its lowest bit lands on bit POS (0 <= POS, POS + K <= 32).
+    template <int POS>
+    __device__ __forceinline__ uint32_t at(const int c) const
+    {
+        const int b = (c % G) * K;
+        const uint32_t w = u[c / G];
+        return (b <= POS ? (w << (POS - b)) : (w >> (b - POS))) & (MASK << POS);
+    }
+
+    // From the tile's packed word stream; p0 = tile-relative index of the lane's first element.
+    __device__ __forceinline__ void from_stream(const uint32_t* wb, const int p0)
+    {
+        if constexpr (POW2 && DPW >= 8) {
+            u[0] = wb[p0 / DPW] >> ((p0 % DPW) * K);
+        } else if constexpr (DPW == 4) {
+            const uint2 w = *reinterpret_cast<const uint2*>(wb + p0 / 4);
+            u[0] = w.x; u[1] = w.y;
+        } else if constexpr (DPW == 2) {
+            const uint4 w = *reinterpret_cast<const uint4*>(wb + p0 / 2);
+            u[0] = w.x; u[1] = w.y; u[2] = w.z; u[3] = w.w;
+        } else {
+            // Words hold DPW fields in their low DPW*K bits.  Two consecutive words, joined
+            // without the unused top bits, always cover a group of G fields.
+#pragma unroll
+            for (int g = 0; g < 8 / G; ++g) {
+                const int p = p0 + g * G, q = p / DPW, f = p - q * DPW;
+                const uint64_t joined = (uint64_t)(wb[q] & (uint32_t)((1ull << (DPW * K)) - 1ull)) |
+                                        ((uint64_t)wb[q + 1] << (DPW * K));
+                u[g] = (uint32_t)(joined >> (f * K));
+            }
+        }
+    }
+
+    // From one Philox call that serves exactly these 8 elements (two draws per word).
+    __device__ __forceinline__ void from_call(const uint4& w)
+    {
+        static_assert(DPW == 2, "a call serves one lane-row only with two draws per word");
+        u[0] = w.x; u[1] = w.y; u[2] = w.z; u[3] = w.w;
+    }
+};
+
+// ----------------------------------------------------------------------------
+// Fast row rounder.  The value is first rescaled by 2^(1 - EMINB) so that the target's
+// exponent range starts where binary32's does: target subnormals become binary32
+// subnormals (the hardware does the alignment shift of Eq. (2)), target normals are
+// scaled exactly, and Eq. (3)-(5) reduce to bfloat16's single addition with
+// sh0 = 24 - P excess bits:  code = (pattern + (n << (sh0 - N))) >> sh0.
+// The multiply rounds toward zero; below the target's emin it keeps 23 - (P - 1) = sh0
+// bits under the target lsb, which is all that SRFF needs for N <= sh0, SRF for
+// N <= sh0 - 1, and (with a sticky bit from a second, upward-rounded multiply) the
+// nearest-even pre-round of SRC for N <= sh0 - 2.  Other (format, N) pairs use round_core.
+// Rows that hold Inf or NaN (or, for bfloat16, |y| > M) are flagged and redone by the caller
+// with round_core: the flag comes from floating-point instructions, off the integer pipe.
+// ----------------------------------------------------------------------------
+template <int FMT, int VAR, int N> struct FastRow {
+    using F = Format<FMT>;
+    static constexpr int SH0 = 24 - F::P;
+    static constexpr bool ALL_BITS = (N == SH0);             // then every variant is exact SR
+    static constexpr bool available =
+        FMT == BF16 ? true
+                    : (VAR == SRFF ? N <= SH0 : VAR == SRF ? N <= SH0 - 1 : N <= SH0 - 2);
+};
+
+template <int FMT, int VAR, int N>
+__device__ __forceinline__ bool round_row_fast(const float (&y)[8], const Draws8<N>& d, uint32_t (&t)[8])
+{
+    using F = Format<FMT>;
+    using R = FastRow<FMT, VAR, N>;
+    constexpr int SH0 = R::SH0;
+    constexpr int EFF = (R::ALL_BITS || (FMT == BF16 && N == 16)) ? SRFF : VAR;
+    constexpr int POS = SH0 - N;                              // where the draw is added
+    float flag = 0.0f;
+#pragma unroll
+    for (int c = 0; c < 8; ++c) {
+        uint32_t u;
+        if constexpr (FMT == BF16) {
+            u = __float_as_uint(y[c]);                        // sign rides along in bit 31
+            // |y| + (maxfloat - M) overflows exactly when |y| > M; Inf and NaN propagate.
+            const float z = __fadd_rn(fabsf(y[c]), __uint_as_float(0x7B7FFF00u));
+            flag = __fmaf_rn(z, 0.0f, flag);
+        } else {
+            const float rescale = __uint_as_float((uint32_t)(128 - F::EMINB) << 23);   // 2^(1 - EMINB)
+            u = __float_as_uint(__fmul_rz(fabsf(y[c]), rescale));
+            if constexpr (EFF == SRC) {
+                const uint32_t up = __float_as_uint(__fmul_ru(fabsf(y[c]), rescale));
+                u |= (u ^ up) & 1u;                           // sticky: round to odd
+            }
+            flag = __fmaf_rn(y[c], 0.0f, flag);               // NaN iff y is Inf or NaN
+        }
+        uint32_t sum;
+        if constexpr (EFF == SRFF) {
+            sum = u + d.template at<POS>(c);
+        } else if constexpr (EFF == SRF) {
+            sum = u + (d.template at<POS>(c) | (1u << (POS - 1)));
+        } else {
+            const uint32_t lsb = (u >> POS) & 1u;
+            sum = u + (d.template at<POS>(c) | ((1u << (POS - 1)) - 1u)) + lsb;
+        }
+        if constexpr (FMT == BF16) t[c] = sum;                // code = bits 16..31
+        else t[c] = min(sum >> SH0, F::MAXCODE);
+    }
+    return flag != flag;
+}
+
 // y = fl32(x * scale); a NaN input passes through so that its sign survives.
 __device__ __forceinline__ uint32_t scaled_bits(float x, float scale)
 {

@@ -104,7 +104,9 @@ __device__ __forceinline__ void store_code1(void* dst, size_t elem, uint32_t c)
 
 // ---------------------------------------------------------------------------- Ops
 // fetch(): issue the loads of 8 consecutive elements; finish(): produce the 8
-// patterns to round (and write back whatever state the op updates);
+// values to round (and write back whatever state the op updates);
+// exact_bits(): the pattern that the element-wise rounder must see for element c
+// (differs from the value's own bits only for NaN, whose sign rule depends on the op);
 // scalar(): the same for one element on the slow path.
 
 struct RoundOp {
@@ -112,12 +114,18 @@ struct RoundOp {
     float scale;
     struct Regs { F8 x; };
     __device__ __forceinline__ void fetch(size_t elem, Regs& r) const { r.x = load_f8_stream(src + elem); }
-    __device__ __forceinline__ void finish(size_t, const Regs& r, uint32_t (&y)[8]) const
+    __device__ __forceinline__ void finish(size_t, const Regs& r, float (&y)[8]) const
     {
         float x[8];
         unpack(r.x, x);
 #pragma unroll
-        for (int c = 0; c < 8; ++c) y[c] = scaled_bits(x[c], scale);
+        for (int c = 0; c < 8; ++c) y[c] = __fmul_rn(x[c], scale);
+    }
+    __device__ __forceinline__ uint32_t exact_bits(const Regs& r, int c, float y) const
+    {
+        float x[8];
+        unpack(r.x, x);
+        return y != y ? __float_as_uint(x[c]) : __float_as_uint(y);   // a NaN keeps the input's sign
     }
     __device__ __forceinline__ uint32_t scalar(size_t i) const { return scaled_bits(src[i], scale); }
 };
@@ -136,14 +144,15 @@ struct SgdOp {
     {
         r.w = load_f8(w + elem); r.g = load_f8_stream(g + elem); r.m = load_f8(m + elem);
     }
-    __device__ __forceinline__ void finish(size_t elem, const Regs& r, uint32_t (&y)[8]) const
+    __device__ __forceinline__ void finish(size_t elem, const Regs& r, float (&y)[8]) const
     {
-        float wv[8], gv[8], mv[8];
-        unpack(r.w, wv); unpack(r.g, gv); unpack(r.m, mv);
+        float gv[8], mv[8];
+        unpack(r.w, y); unpack(r.g, gv); unpack(r.m, mv);
 #pragma unroll
-        for (int c = 0; c < 8; ++c) { step(wv[c], gv[c], mv[c]); y[c] = arith_bits(wv[c]); }
-        store_f8(w + elem, wv); store_f8(m + elem, mv);
+        for (int c = 0; c < 8; ++c) step(y[c], gv[c], mv[c]);
+        store_f8(w + elem, y); store_f8(m + elem, mv);
     }
+    __device__ __forceinline__ uint32_t exact_bits(const Regs&, int, float y) const { return arith_bits(y); }
     __device__ __forceinline__ uint32_t scalar(size_t i) const
     {
         float wv = w[i], mv = m[i];
@@ -170,14 +179,15 @@ struct AdamOp {
         r.w = load_f8(w + elem); r.g = load_f8_stream(g + elem);
         r.m = load_f8(m + elem); r.v = load_f8(v + elem);
     }
-    __device__ __forceinline__ void finish(size_t elem, const Regs& r, uint32_t (&y)[8]) const
+    __device__ __forceinline__ void finish(size_t elem, const Regs& r, float (&y)[8]) const
     {
-        float wv[8], gv[8], mv[8], vv[8];
-        unpack(r.w, wv); unpack(r.g, gv); unpack(r.m, mv); unpack(r.v, vv);
+        float gv[8], mv[8], vv[8];
+        unpack(r.w, y); unpack(r.g, gv); unpack(r.m, mv); unpack(r.v, vv);
 #pragma unroll
-        for (int c = 0; c < 8; ++c) { step(wv[c], gv[c], mv[c], vv[c]); y[c] = arith_bits(wv[c]); }
-        store_f8(w + elem, wv); store_f8(m + elem, mv); store_f8(v + elem, vv);
+        for (int c = 0; c < 8; ++c) step(y[c], gv[c], mv[c], vv[c]);
+        store_f8(w + elem, y); store_f8(m + elem, mv); store_f8(v + elem, vv);
     }
+    __device__ __forceinline__ uint32_t exact_bits(const Regs&, int, float y) const { return arith_bits(y); }
     __device__ __forceinline__ uint32_t scalar(size_t i) const
     {
         float wv = w[i], mv = m[i], vv = v[i];
@@ -202,7 +212,8 @@ struct AccumOp {
             r.c = make_uint4(t.x, t.y, 0u, 0u);
         }
     }
-    __device__ __forceinline__ void finish(size_t, const Regs& r, uint32_t (&y)[8]) const
+    __device__ __forceinline__ uint32_t exact_bits(const Regs&, int, float y) const { return arith_bits(y); }
+    __device__ __forceinline__ void finish(size_t, const Regs& r, float (&y)[8]) const
     {
         float uv[8];
         unpack(r.u, uv);
@@ -212,7 +223,7 @@ struct AccumOp {
             uint32_t code;
             if constexpr (Format<FMT>::K == 16) code = (cw[c >> 1] >> ((c & 1) * 16)) & 0xFFFFu;
             else code = (cw[c >> 2] >> ((c & 3) * 8)) & 0xFFu;
-            y[c] = arith_bits(__fadd_rn(decode_element<FMT>(code), uv[c]));
+            y[c] = __fadd_rn(decode_element<FMT>(code), uv[c]);
         }
     }
     __device__ __forceinline__ uint32_t scalar(size_t i) const
@@ -224,42 +235,37 @@ struct AccumOp {
     }
 };
 
-// ---------------------------------------------------------------------------- draws from a word buffer
-// wb: the tile's packed word stream; p0: tile-relative index of the lane's first element (multiple of 8).
-template <int K>
-__device__ __forceinline__ void draws8(const uint32_t* wb, int p0, uint32_t (&n)[8])
+// ---------------------------------------------------------------------------- packing a row of codes
+// Fast rows: t[] as left by round_row_fast (bfloat16: code in bits 16..31 with the sign;
+// other formats: magnitude code, sign still to be taken from y).
+template <int FMT>
+__device__ __forceinline__ void store_row_fast(void* dst, size_t elem, const uint32_t (&t)[8], const float (&y)[8])
 {
-    using T = Tile<K>;
-    constexpr int DPW = T::DPW;
-    if constexpr (DPW >= 8 && (DPW & (DPW - 1)) == 0) {
-        const uint32_t w = wb[p0 / DPW] >> ((p0 % DPW) * K);          // all 8 fields sit in one word
+    if constexpr (FMT == BF16) {
+        uint4 v;
+        v.x = __byte_perm(t[0], t[1], 0x7632); v.y = __byte_perm(t[2], t[3], 0x7632);
+        v.z = __byte_perm(t[4], t[5], 0x7632); v.w = __byte_perm(t[6], t[7], 0x7632);
+        __stcs(reinterpret_cast<uint4*>(static_cast<uint16_t*>(dst) + elem), v);
+    } else if constexpr (Format<FMT>::K == 16) {
+        uint32_t o[4];
 #pragma unroll
-        for (int c = 0; c < 8; ++c) n[c] = (w >> (c * K)) & T::MASK;
-    } else if constexpr (DPW == 4) {
-        const uint2 w = *reinterpret_cast<const uint2*>(wb + p0 / 4);
-#pragma unroll
-        for (int c = 0; c < 8; ++c) n[c] = ((c < 4 ? w.x : w.y) >> ((c & 3) * K)) & T::MASK;
-    } else if constexpr (DPW == 2) {
-        const uint4 w = *reinterpret_cast<const uint4*>(wb + p0 / 2);
-        const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
-#pragma unroll
-        for (int c = 0; c < 8; ++c) n[c] = (ww[c >> 1] >> ((c & 1) * K)) & T::MASK;
-    } else {
-#pragma unroll
-        for (int c = 0; c < 8; ++c) {
-            const int p = p0 + c, q = p / DPW, f = p - q * DPW;
-            n[c] = (wb[q] >> (f * K)) & T::MASK;
+        for (int j = 0; j < 4; ++j) {
+            const uint32_t signs = __byte_perm(__float_as_uint(y[2 * j]), __float_as_uint(y[2 * j + 1]), 0x7632);
+            o[j] = (t[2 * j] + t[2 * j + 1] * 65536u) | (signs & 0x80008000u);
         }
-    }
-}
-
-template <int K>
-__device__ __forceinline__ void draws8_from_call(const uint4& w, uint32_t (&n)[8])
-{
-    static_assert(Tile<K>::DPW == 2, "one Philox call per 8 elements only with two draws per word");
-    const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+        __stcs(reinterpret_cast<uint4*>(static_cast<uint16_t*>(dst) + elem), make_uint4(o[0], o[1], o[2], o[3]));
+    } else {
+        uint32_t o[2];
 #pragma unroll
-    for (int c = 0; c < 8; ++c) n[c] = (ww[c >> 1] >> ((c & 1) * K)) & Tile<K>::MASK;
+        for (int j = 0; j < 2; ++j) {
+            const uint32_t s01 = __byte_perm(__float_as_uint(y[4 * j]), __float_as_uint(y[4 * j + 1]), 0x7373);
+            const uint32_t s23 = __byte_perm(__float_as_uint(y[4 * j + 2]), __float_as_uint(y[4 * j + 3]), 0x7373);
+            const uint32_t signs = __byte_perm(s01, s23, 0x5410);
+            o[j] = (t[4 * j] + t[4 * j + 1] * 256u + t[4 * j + 2] * 65536u + t[4 * j + 3] * 16777216u) |
+                   (signs & 0x80808080u);
+        }
+        __stcs(reinterpret_cast<uint2*>(static_cast<uint8_t*>(dst) + elem), make_uint2(o[0], o[1]));
+    }
 }
 
 // ---------------------------------------------------------------------------- the bandwidth kernel
@@ -273,7 +279,7 @@ tile_kernel(const Op op, void* __restrict__ dst, const uint64_t n_tiles, const u
 {
     using T = Tile<K>;
     constexpr bool OWN_CALL = (T::DPW == 2) && !BITS;      // a call serves exactly one lane-row
-    __shared__ __align__(16) uint32_t wordbuf[WARPS_PER_CTA][OWN_CALL ? 4 : T::WORDS];
+    __shared__ __align__(16) uint32_t wordbuf[WARPS_PER_CTA][OWN_CALL ? 4 : T::WORDS + 4];   // +4: the joined-word read of the last group
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     uint32_t* wb = wordbuf[warp];
 
@@ -306,17 +312,26 @@ tile_kernel(const Op op, void* __restrict__ dst, const uint64_t n_tiles, const u
             for (int j = 0; j < 4; ++j) {
                 if (rb + j < T::ROWS) {
                     const int p0 = (rb + j) * ROW_ELEMS + lane * 8;
-                    uint32_t y[8], n[8], c[8];
+                    float y[8];
                     op.finish(e0 + p0, regs[j], y);
-                    if constexpr (OWN_CALL) {
-                        const uint4 w = philox_block(tile_call0 + (rb + j) * 32 + lane, k0, k1);
-                        draws8_from_call<K>(w, n);
-                    } else {
-                        draws8<K>(wb, p0, n);
+                    Draws8<K> d;
+                    if constexpr (OWN_CALL) d.from_call(philox_block(tile_call0 + (rb + j) * 32 + lane, k0, k1));
+                    else d.from_stream(wb, p0);
+                    bool redo = true;
+                    if constexpr (FastRow<FMT, VAR, K>::available) {
+                        uint32_t t[8];
+                        redo = round_row_fast<FMT, VAR, K>(y, d, t);
+                        if (!redo) store_row_fast<FMT>(dst, e0 + p0, t, y);
                     }
+                    if (redo) {
+                        // a special value in this lane's row (rare), or a (format, k) pair without a fast form
+                        uint32_t c[8];
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) c[i] = round_core<FMT, false>(y[i], n[i], VAR, K, nullptr);
-                    store_codes8<FMT>(dst, e0 + p0, c);
+                        for (int i = 0; i < 8; ++i)
+                            c[i] = round_core<FMT, false>(op.exact_bits(regs[j], i, y[i]), d.template at<0>(i), VAR, K,
+                                                          nullptr);
+                        store_codes8<FMT>(dst, e0 + p0, c);
+                    }
                 }
             }
         }
