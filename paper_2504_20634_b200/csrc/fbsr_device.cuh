@@ -166,6 +166,13 @@ template <int K> struct Draws8 {
         return (b <= POS ? (w << (POS - b)) : (w >> (b - POS))) & (MASK << POS);
     }
 
+    // Field of element c without its S lowest bits, at bit 0.
+    template <int S>
+    __device__ __forceinline__ uint32_t top(const int c) const
+    {
+        return (u[c / G] >> ((c % G) * K + S)) & (MASK >> S);
+    }
+
     // From the tile's packed word stream; p0 = tile-relative index of the lane's first element.
     __device__ __forceinline__ void from_stream(const uint32_t* wb, const int p0)
     {
@@ -207,7 +214,14 @@ template <int K> struct Draws8 {
 // The multiply rounds toward zero; below the target's emin it keeps 23 - (P - 1) = sh0
 // bits under the target lsb, which is all that SRFF needs for N <= sh0, SRF for
 // N <= sh0 - 1, and (with a sticky bit from a second, upward-rounded multiply) the
-// nearest-even pre-round of SRC for N <= sh0 - 2.  Other (format, N) pairs use round_core.
+// nearest-even pre-round of SRC for N <= sh0 - 2.
+// For larger N (binary16 with N >= 12..14) the subnormal range needs more bits than the
+// rescaled pattern keeps, so two candidates are formed and one selected per element:
+//   |y| >= 2^emin : the pattern form; with N >= sh0 it is exact SR on the sh0 excess bits,
+//                   which only the top sh0 bits of the draw can influence;
+//   |y| <  2^emin : sigma~ 2^N = |y| / 2^(emin - (P-1) - N) converted to an integer (toward
+//                   zero for SRFF/SRF, to nearest-even for SRC's pre-round), draw added,
+//                   N bits dropped; the biased exponent is 0, so sigma is the code.
 // Rows that hold Inf or NaN (or, for bfloat16, |y| > M) are flagged and redone by the caller
 // with round_core: the flag comes from floating-point instructions, off the integer pipe.
 // ----------------------------------------------------------------------------
@@ -215,7 +229,7 @@ template <int FMT, int VAR, int N> struct FastRow {
     using F = Format<FMT>;
     static constexpr int SH0 = 24 - F::P;
     static constexpr bool ALL_BITS = (N == SH0);             // then every variant is exact SR
-    static constexpr bool available =
+    static constexpr bool one_regime =
         FMT == BF16 ? true
                     : (VAR == SRFF ? N <= SH0 : VAR == SRF ? N <= SH0 - 1 : N <= SH0 - 2);
 };
@@ -229,6 +243,32 @@ __device__ __forceinline__ bool round_row_fast(const float (&y)[8], const Draws8
     constexpr int EFF = (R::ALL_BITS || (FMT == BF16 && N == 16)) ? SRFF : VAR;
     constexpr int POS = SH0 - N;                              // where the draw is added
     float flag = 0.0f;
+    if constexpr (!R::one_regime) {
+        static_assert(FMT != BF16 && N >= SH0 - 1, "two-regime form is for draws about as wide as the excess bits");
+        const float rescale = __uint_as_float((uint32_t)(128 - F::EMINB) << 23);        // 2^(1 - EMINB)
+        const float min_normal = __uint_as_float((uint32_t)F::EMINB << 23);             // 2^emin
+        constexpr int EXTRA = (VAR == SRF) ? 1 : 0;                                     // SRF compares half a step finer
+        const float to_steps = __uint_as_float((uint32_t)(F::P + N + EXTRA + 253 - F::EMINB) << 23);
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+            const float a = fabsf(y[c]);
+            flag = __fmaf_rn(y[c], 0.0f, flag);
+            // normal range of the target
+            const uint32_t u = __float_as_uint(__fmul_rz(a, rescale));
+            uint32_t sum;
+            if constexpr (N >= SH0) sum = u + d.template top<N - SH0>(c);
+            else sum = u + d.template at<1>(c) + ((u >> 1) & 1u);                       // SRC, N = sh0 - 1
+            const uint32_t hi = min(sum >> SH0, F::MAXCODE);
+            // subnormal range of the target
+            const float steps = __fmul_rn(a, to_steps);                                 // exact below 2^emin
+            uint32_t lo;
+            if constexpr (VAR == SRFF) lo = (__float2uint_rz(steps) + d.template at<0>(c)) >> N;
+            else if constexpr (VAR == SRF) lo = (__float2uint_rz(steps) + ((d.template at<0>(c) << 1) | 1u)) >> (N + 1);
+            else lo = (__float2uint_rn(steps) + d.template at<0>(c)) >> N;
+            t[c] = a < min_normal ? lo : hi;
+        }
+        return flag != flag;
+    } else {
 #pragma unroll
     for (int c = 0; c < 8; ++c) {
         uint32_t u;
@@ -259,6 +299,7 @@ __device__ __forceinline__ bool round_row_fast(const float (&y)[8], const Draws8
         else t[c] = min(sum >> SH0, F::MAXCODE);
     }
     return flag != flag;
+    }
 }
 
 // y = fl32(x * scale); a NaN input passes through so that its sign survives.

@@ -46,15 +46,11 @@ int launch_tiles(const Op& op, const CallArgs& a, const Plan& p)
 {
     using T = Tile<K>;
     auto kern = tile_kernel<Op, FMT, VAR, K, BITS>;
-    static int ctas_per_sm = 0;
-    if (ctas_per_sm == 0) {
-        int occ = 0;
-        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kern, CTA_THREADS, 0) != cudaSuccess || occ < 1) occ = 1;
-        ctas_per_sm = occ;
-    }
+    // One tile per warp, CTAs handed out by the hardware scheduler.  A persistent grid with a static
+    // tile stride measured 5-10 % slower here: multiprocessors do not all see the same memory
+    // bandwidth, and a static split makes the whole launch wait for the slowest of them.
     const uint64_t want = (p.n_tiles + WARPS_PER_CTA - 1) / WARPS_PER_CTA;
-    const uint64_t cap = (uint64_t)sm_count() * ctas_per_sm;
-    const unsigned grid = (unsigned)(want < cap ? want : cap);
+    const unsigned grid = (unsigned)(want < 0x7FFFFFFFull ? want : 0x7FFFFFFFull);
     const Op adv = op_advance(op, p.head);
     void* dst = static_cast<char*>(a.dst) + p.head * CODE_BYTES;
     const uint64_t call0 = BITS ? 0 : (a.offset + p.head) / T::E;

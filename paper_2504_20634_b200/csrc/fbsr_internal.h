@@ -42,6 +42,5 @@ FBSR_DECLARE_DISPATCH(0) FBSR_DECLARE_DISPATCH(1) FBSR_DECLARE_DISPATCH(2) FBSR_
 #undef FBSR_DECLARE_DISPATCH
 
 void count_launch();                         // bumps the counter behind fbsr_launch_count()
-int sm_count();                              // multiprocessors of the current device
 
 }  // namespace fbsr

@@ -25,7 +25,15 @@
 
 namespace fbsr {
 
-constexpr int WARPS_PER_CTA = 8;
+// Tuning constants (overridable at compile time for experiments).
+#ifndef FBSR_WARPS_PER_CTA
+#define FBSR_WARPS_PER_CTA 8
+#endif
+#ifndef FBSR_ROW_BATCH
+#define FBSR_ROW_BATCH 4            // rows whose loads are issued before the first row is consumed
+#endif
+constexpr int WARPS_PER_CTA = FBSR_WARPS_PER_CTA;
+constexpr int ROW_BATCH = FBSR_ROW_BATCH;
 constexpr int CTA_THREADS = WARPS_PER_CTA * 32;
 constexpr int ROW_ELEMS = 256;          // 32 lanes x 8 elements
 
@@ -110,6 +118,7 @@ __device__ __forceinline__ void store_code1(void* dst, size_t elem, uint32_t c)
 // scalar(): the same for one element on the slow path.
 
 struct RoundOp {
+    static constexpr int BATCH = ROW_BATCH;
     const float* src;
     float scale;
     struct Regs { F8 x; };
@@ -132,6 +141,7 @@ struct RoundOp {
 
 // m' = fma(mu, m, g);  w' = fma(-lr, m', w)
 struct SgdOp {
+    static constexpr int BATCH = ROW_BATCH >= 2 ? ROW_BATCH / 2 : 1;
     float* w; const float* g; float* m;
     float neg_lr, mu;
     struct Regs { F8 w, g, m; };
@@ -164,6 +174,7 @@ struct SgdOp {
 
 // m' = fma(b1, m, a1 g); v' = fma(b2, v, (a2 g) g); d = sqrt(v') c2 + eps; w' = fma(-c1, m'/d, w)
 struct AdamOp {
+    static constexpr int BATCH = ROW_BATCH >= 2 ? ROW_BATCH / 2 : 1;
     float* w; const float* g; float* m; float* v;
     float beta1, beta2, eps, neg_c1, c2, a1, a2;
     struct Regs { F8 w, g, m, v; };
@@ -200,6 +211,7 @@ struct AdamOp {
 // y = fl32(value(w_lp) + u); the codes are rewritten in place by the caller of finish()
 template <int FMT>
 struct AccumOp {
+    static constexpr int BATCH = ROW_BATCH;
     const void* w_lp; const float* u;
     struct Regs { F8 u; uint4 c; };
     __device__ __forceinline__ void fetch(size_t elem, Regs& r) const
@@ -269,7 +281,8 @@ __device__ __forceinline__ void store_row_fast(void* dst, size_t elem, const uin
 }
 
 // ---------------------------------------------------------------------------- the bandwidth kernel
-// Elements [0, n_tiles * ELEMS) relative to the pointers held by op/dst.
+// Elements [0, n_tiles * ELEMS) relative to the pointers held by op/dst.  Normally launched with one
+// tile per warp; the loop only matters when the grid had to be capped.
 // call0: global index of the Philox call that serves element 0 (Philox source), or
 // words: the packed word stream whose word 0 serves element 0 (supplied bits).
 template <class Op, int FMT, int VAR, int K, bool BITS>
@@ -303,13 +316,15 @@ tile_kernel(const Op op, void* __restrict__ dst, const uint64_t n_tiles, const u
         }
 
 #pragma unroll
-        for (int rb = 0; rb < T::ROWS; rb += 4) {
-            typename Op::Regs regs[4];
+        constexpr int BATCH = Op::BATCH < T::ROWS ? Op::BATCH : T::ROWS;
 #pragma unroll
-            for (int j = 0; j < 4; ++j)
+        for (int rb = 0; rb < T::ROWS; rb += BATCH) {
+            typename Op::Regs regs[BATCH];
+#pragma unroll
+            for (int j = 0; j < BATCH; ++j)
                 if (rb + j < T::ROWS) op.fetch(e0 + (rb + j) * ROW_ELEMS + lane * 8, regs[j]);
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
+            for (int j = 0; j < BATCH; ++j) {
                 if (rb + j < T::ROWS) {
                     const int p0 = (rb + j) * ROW_ELEMS + lane * 8;
                     float y[8];
@@ -317,14 +332,12 @@ tile_kernel(const Op op, void* __restrict__ dst, const uint64_t n_tiles, const u
                     Draws8<K> d;
                     if constexpr (OWN_CALL) d.from_call(philox_block(tile_call0 + (rb + j) * 32 + lane, k0, k1));
                     else d.from_stream(wb, p0);
-                    bool redo = true;
-                    if constexpr (FastRow<FMT, VAR, K>::available) {
-                        uint32_t t[8];
-                        redo = round_row_fast<FMT, VAR, K>(y, d, t);
-                        if (!redo) store_row_fast<FMT>(dst, e0 + p0, t, y);
-                    }
-                    if (redo) {
-                        // a special value in this lane's row (rare), or a (format, k) pair without a fast form
+                    uint32_t t[8];
+                    const bool redo = round_row_fast<FMT, VAR, K>(y, d, t);
+                    if (!redo) {
+                        store_row_fast<FMT>(dst, e0 + p0, t, y);
+                    } else {
+                        // a special value somewhere in this lane's row (rare): element-wise, exact
                         uint32_t c[8];
 #pragma unroll
                         for (int i = 0; i < 8; ++i)
