@@ -158,7 +158,7 @@ def main():
         return
 
     import paper_2504_20634_b200 as fbsr            # raises if libfbsr.so is missing: no fallback
-    from paper_2504_20634_b200 import workloads
+    from paper_2504_20634_b200 import sharding, workloads
 
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
@@ -172,10 +172,12 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
-    # ---- inputs: this rank's shard of the sweep tensor (global index = rank * N_ELEMS + i)
-    offset = rank * N_ELEMS
-    x = workloads.bandwidth_sweep(N_ELEMS, seed=SEED + rank, device=dev)
-    out = torch.empty(N_ELEMS, dtype=torch.uint16, device=dev)
+    # ---- inputs: this rank's shard of a world * 2^28 element tensor (weak scaling); shard boundaries sit
+    # on a multiple of every tile size, global index of local element i = offset + i
+    offset, shard_end = sharding.my_shard(world * N_ELEMS, rank, world)
+    n_local = shard_end - offset
+    x = workloads.bandwidth_sweep(n_local, seed=SEED + rank, device=dev)
+    out = torch.empty(n_local, dtype=torch.uint16, device=dev)
     combos = sweep()
     stream = torch.cuda.current_stream(dev)
 
@@ -199,24 +201,19 @@ def main():
     launches = fbsr.fbsr_launch_count() - launches0
     clocks = sampler.stop()
     ms = ev0.elapsed_time(ev1)
-    if dist is not None:
-        t = torch.tensor([ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
-        lt = torch.tensor([launches], device=dev, dtype=torch.int64)
-        dist.all_reduce(lt)
-        launches = int(lt.item())
+    ms = sharding.max_over_ranks(ms, dist, dev)
+    launches = int(sharding.sum_over_ranks(int(launches), dist, dev))
     ms_per_step = ms / args.steps
     total_elems = float(N_ELEMS) * len(combos) * world
     value = total_elems / (ms_per_step * 1e-3) / 1e9
 
     # ---- roofline of the tiled rounding kernel: all 48 launches move 6 B/element
     peak, peak_kind = measured_peak_gbs()
-    achieved = BYTES_PER_ELEM * N_ELEMS * len(combos) / (ms_per_step * 1e-3) / 1e9
+    achieved = BYTES_PER_ELEM * n_local * len(combos) / (ms_per_step * 1e-3) / 1e9
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                 "traffic": None, "peak_source": peak_kind + " copy bandwidth",
                 "kernel": "fbsr::tile_kernel<RoundOp, fmt, variant, k> (average over the 48 launches of a step)",
-                "algorithmic_bytes_per_launch": BYTES_PER_ELEM * N_ELEMS,
+                "algorithmic_bytes_per_launch": BYTES_PER_ELEM * n_local,
                 "frac_of_8TBps": achieved / 8000.0}
 
     # ---- end to end through the host-buffer entry point (pinned host memory, copies inside the timed region)
@@ -248,10 +245,7 @@ def main():
         t1.record(stream)
         barrier()
         e_ms = t0.elapsed_time(t1)
-        if dist is not None:
-            t = torch.tensor([e_ms], device=dev, dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e_ms = float(t.item())
+        e_ms = sharding.max_over_ranks(e_ms, dist, dev)
         e_val = float(n_e2e) * len(e2e_combos) * e2e_steps * world / (e_ms * 1e-3) / 1e9
         e2e = {"value": e_val, "unit": UNIT, "h2d_bytes_per_step": 4 * n_e2e * len(e2e_combos),
                "d2h_bytes_per_step": 2 * n_e2e * len(e2e_combos),
@@ -271,7 +265,7 @@ def main():
             evs.append((fmt, variant, k, a, b))
         torch.cuda.synchronize()
         for fmt, variant, k, a, b in evs:
-            table["%s/%s/k%d" % (fmt, variant, k)] = round(BYTES_PER_ELEM * N_ELEMS / (a.elapsed_time(b) / 3 * 1e-3) / 1e9, 1)
+            table["%s/%s/k%d" % (fmt, variant, k)] = round(BYTES_PER_ELEM * n_local / (a.elapsed_time(b) / 3 * 1e-3) / 1e9, 1)
         extras["round_GBps"] = table
         # fp8 leg of the metric (5 B/element), 2^27 elements
         x8 = x[: 1 << 27]
