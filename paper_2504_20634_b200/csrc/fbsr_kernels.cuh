@@ -29,6 +29,15 @@ namespace fbsr {
 #ifndef FBSR_WARPS_PER_CTA
 #define FBSR_WARPS_PER_CTA 8
 #endif
+#ifndef FBSR_MIN_CTAS_ROUND
+#define FBSR_MIN_CTAS_ROUND 4       // resident CTAs the compiler must allow (caps registers at 64)
+#endif
+#ifndef FBSR_MIN_CTAS_SGD
+#define FBSR_MIN_CTAS_SGD 2
+#endif
+#ifndef FBSR_MIN_CTAS_ADAM
+#define FBSR_MIN_CTAS_ADAM 2
+#endif
 #ifndef FBSR_ROW_BATCH
 #define FBSR_ROW_BATCH 4            // rows whose loads are issued before the first row is consumed
 #endif
@@ -40,14 +49,16 @@ constexpr int ROW_ELEMS = 256;          // 32 lanes x 8 elements
 template <int K> struct Tile {
     static constexpr int DPW = 32 / K;                        // draws per word
     static constexpr int E = 4 * DPW;                         // elements per Philox call
-    static constexpr int R0 = (DPW % 2 == 0) ? DPW / 2 : DPW; // rows holding 32 (or 64) whole calls
-    static constexpr int MULT = R0 >= 4 ? 1 : (4 + R0 - 1) / R0;
-    static constexpr int ROWS = R0 * MULT;
+    static constexpr bool POW2 = (DPW & (DPW - 1)) == 0;
+    // Power-of-two dpw: 4 rows (1024 elements) always hold whole calls.  Otherwise the smallest
+    // number of rows that does (dpw rows, or dpw/2 when dpw is even), doubled while below 4.
+    static constexpr int R0 = (DPW % 2 == 0) ? DPW / 2 : DPW;
+    static constexpr int ROWS = POW2 ? 4 : (R0 >= 4 ? R0 : R0 * ((4 + R0 - 1) / R0));
     static constexpr int ELEMS = ROWS * ROW_ELEMS;
     static constexpr int CALLS = ELEMS / E;                   // Philox calls per tile
     static constexpr int WORDS = ELEMS / DPW;                 // random words per tile
     static constexpr uint32_t MASK = (1u << K) - 1u;
-    static_assert(ELEMS % E == 0 && CALLS % 32 == 0, "tile must hold whole calls, evenly per lane");
+    static_assert(ELEMS % E == 0, "a tile must hold whole Philox calls");
 };
 
 // ---------------------------------------------------------------------------- vector memory access
@@ -118,7 +129,7 @@ __device__ __forceinline__ void store_code1(void* dst, size_t elem, uint32_t c)
 // scalar(): the same for one element on the slow path.
 
 struct RoundOp {
-    static constexpr int BATCH = ROW_BATCH;
+    static constexpr int BATCH = ROW_BATCH, MIN_CTAS = FBSR_MIN_CTAS_ROUND;
     const float* src;
     float scale;
     struct Regs { F8 x; };
@@ -141,7 +152,7 @@ struct RoundOp {
 
 // m' = fma(mu, m, g);  w' = fma(-lr, m', w)
 struct SgdOp {
-    static constexpr int BATCH = ROW_BATCH >= 2 ? ROW_BATCH / 2 : 1;
+    static constexpr int BATCH = ROW_BATCH >= 2 ? ROW_BATCH / 2 : 1, MIN_CTAS = FBSR_MIN_CTAS_SGD;
     float* w; const float* g; float* m;
     float neg_lr, mu;
     struct Regs { F8 w, g, m; };
@@ -174,7 +185,7 @@ struct SgdOp {
 
 // m' = fma(b1, m, a1 g); v' = fma(b2, v, (a2 g) g); d = sqrt(v') c2 + eps; w' = fma(-c1, m'/d, w)
 struct AdamOp {
-    static constexpr int BATCH = ROW_BATCH >= 2 ? ROW_BATCH / 2 : 1;
+    static constexpr int BATCH = ROW_BATCH >= 2 ? ROW_BATCH / 2 : 1, MIN_CTAS = FBSR_MIN_CTAS_ADAM;
     float* w; const float* g; float* m; float* v;
     float beta1, beta2, eps, neg_c1, c2, a1, a2;
     struct Regs { F8 w, g, m, v; };
@@ -211,7 +222,7 @@ struct AdamOp {
 // y = fl32(value(w_lp) + u); the codes are rewritten in place by the caller of finish()
 template <int FMT>
 struct AccumOp {
-    static constexpr int BATCH = ROW_BATCH;
+    static constexpr int BATCH = ROW_BATCH, MIN_CTAS = FBSR_MIN_CTAS_ROUND;
     const void* w_lp; const float* u;
     struct Regs { F8 u; uint4 c; };
     __device__ __forceinline__ void fetch(size_t elem, Regs& r) const
@@ -286,7 +297,7 @@ __device__ __forceinline__ void store_row_fast(void* dst, size_t elem, const uin
 // call0: global index of the Philox call that serves element 0 (Philox source), or
 // words: the packed word stream whose word 0 serves element 0 (supplied bits).
 template <class Op, int FMT, int VAR, int K, bool BITS>
-__global__ void __launch_bounds__(CTA_THREADS)
+__global__ void __launch_bounds__(CTA_THREADS, Op::MIN_CTAS)
 tile_kernel(const Op op, void* __restrict__ dst, const uint64_t n_tiles, const uint64_t call0,
             const uint32_t k0, const uint32_t k1, const uint32_t* __restrict__ words)
 {
@@ -305,18 +316,22 @@ tile_kernel(const Op op, void* __restrict__ dst, const uint64_t n_tiles, const u
             const uint32_t* src_words = words + tile * T::WORDS;
 #pragma unroll
             for (int j = 0; j < T::WORDS / 32; ++j) wb[j * 32 + lane] = __ldg(src_words + j * 32 + lane);
+            static_assert(T::WORDS % 32 == 0, "whole warp-rows of words");
             __syncwarp();
         } else if constexpr (!OWN_CALL) {
 #pragma unroll
-            for (int j = 0; j < T::CALLS / 32; ++j) {
+            for (int j = 0; j < (T::CALLS + 31) / 32; ++j) {
                 const int c = j * 32 + lane;
-                *reinterpret_cast<uint4*>(wb + 4 * c) = philox_block(tile_call0 + c, k0, k1);
+                if (T::CALLS % 32 == 0 || c < T::CALLS)
+                    *reinterpret_cast<uint4*>(wb + 4 * c) = philox_block(tile_call0 + c, k0, k1);
             }
             __syncwarp();
         }
 
 #pragma unroll
-        constexpr int BATCH = Op::BATCH < T::ROWS ? Op::BATCH : T::ROWS;
+        // rows are taken in equal batches of at most Op::BATCH (5 rows: 3 + 2, not 4 + 1)
+        constexpr int N_BATCHES = (T::ROWS + Op::BATCH - 1) / Op::BATCH;
+        constexpr int BATCH = (T::ROWS + N_BATCHES - 1) / N_BATCHES;
 #pragma unroll
         for (int rb = 0; rb < T::ROWS; rb += BATCH) {
             typename Op::Regs regs[BATCH];

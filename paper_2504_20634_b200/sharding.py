@@ -11,6 +11,8 @@ import math
 def tile_elements(k_bits):
     """Elements per warp tile of the fast path (mirrors fbsr_tile_elements of the library)."""
     dpw = 32 // k_bits
+    if dpw & (dpw - 1) == 0:
+        return 1024
     rows = dpw // 2 if dpw % 2 == 0 else dpw
     if rows < 4:
         rows *= -(-4 // rows)
