@@ -49,14 +49,15 @@ int launch_tiles(const Op& op, const CallArgs& a, const Plan& p)
     // One tile per warp, CTAs handed out by the hardware scheduler.  A persistent grid with a static
     // tile stride measured 5-10 % slower here: multiprocessors do not all see the same memory
     // bandwidth, and a static split makes the whole launch wait for the slowest of them.
+    const uint32_t tail_count = (uint32_t)(a.n - p.tail_begin);          // < one tile; served by an extra CTA
     const uint64_t want = (p.n_tiles + WARPS_PER_CTA - 1) / WARPS_PER_CTA;
-    const unsigned grid = (unsigned)(want < 0x7FFFFFFFull ? want : 0x7FFFFFFFull);
+    const unsigned grid = (unsigned)(want < 0x7FFFFFF0ull ? want : 0x7FFFFFF0ull) + (tail_count ? 1u : 0u);
     const Op adv = op_advance(op, p.head);
     void* dst = static_cast<char*>(a.dst) + p.head * CODE_BYTES;
     const uint64_t call0 = BITS ? 0 : (a.offset + p.head) / T::E;
     const uint32_t* words = BITS ? a.words + p.head / T::DPW : nullptr;
     kern<<<grid, CTA_THREADS, 0, a.stream>>>(adv, dst, p.n_tiles, call0, (uint32_t)a.seed,
-                                             (uint32_t)(a.seed >> 32), words);
+                                             (uint32_t)(a.seed >> 32), words, tail_count);
     count_launch();
     return 0;
 }
@@ -81,7 +82,7 @@ int launch_generic(const Op& op, const CallArgs& a, size_t i_begin, size_t i_end
     return 0;
 }
 
-// Split a call into [0, head) slow, whole tiles fast, [tail_begin, n) slow.
+// Split a call into [0, head) on the general kernel, whole tiles, and [tail_begin, n) (less than a tile).
 template <class Op, int K, bool BITS>
 Plan make_plan(const Op& op, const CallArgs& a)
 {
@@ -106,8 +107,7 @@ int run(const Op& op, const CallArgs& a)
     const Plan p = make_plan<Op, K, BITS>(op, a);
     if (p.n_tiles == 0) return launch_generic<Op, BITS, false>(op, a, 0, a.n, nullptr);
     launch_generic<Op, BITS, false>(op, a, 0, p.head, nullptr);
-    launch_tiles<Op, VAR, K, BITS>(op, a, p);
-    launch_generic<Op, BITS, false>(op, a, p.tail_begin, a.n, nullptr);
+    launch_tiles<Op, VAR, K, BITS>(op, a, p);          // whole tiles and the ragged end
     return 0;
 }
 

@@ -299,16 +299,37 @@ __device__ __forceinline__ void store_row_fast(void* dst, size_t elem, const uin
 template <class Op, int FMT, int VAR, int K, bool BITS>
 __global__ void __launch_bounds__(CTA_THREADS, Op::MIN_CTAS)
 tile_kernel(const Op op, void* __restrict__ dst, const uint64_t n_tiles, const uint64_t call0,
-            const uint32_t k0, const uint32_t k1, const uint32_t* __restrict__ words)
+            const uint32_t k0, const uint32_t k1, const uint32_t* __restrict__ words, const uint32_t tail_count)
 {
     using T = Tile<K>;
+    // The elements after the last whole tile (fewer than one tile) are done by CTA 0, one element per
+    // thread and step, each with its own generator call: it starts first and overlaps the tiles.
+    const uint32_t first_tile_cta = tail_count ? 1u : 0u;
+    if (tail_count && blockIdx.x == 0) {
+        const size_t tail_begin = (size_t)n_tiles * T::ELEMS;
+        for (uint32_t i = threadIdx.x; i < tail_count; i += CTA_THREADS) {
+            const size_t p = tail_begin + i;
+            const uint32_t j = (uint32_t)(p % T::E);
+            uint32_t word;
+            if constexpr (BITS) {
+                word = words[p / T::DPW];
+            } else {
+                const uint4 o = philox_block(call0 + p / T::E, k0, k1);
+                const uint32_t ws = j / T::DPW;
+                word = ws == 0 ? o.x : ws == 1 ? o.y : ws == 2 ? o.z : o.w;
+            }
+            const uint32_t n = (word >> ((j % T::DPW) * K)) & T::MASK;
+            store_code1<FMT>(dst, p, round_core<FMT, false>(op.scalar(p), n, VAR, K, nullptr));
+        }
+        return;
+    }
     constexpr bool OWN_CALL = (T::DPW == 2) && !BITS;      // a call serves exactly one lane-row
     __shared__ __align__(16) uint32_t wordbuf[WARPS_PER_CTA][OWN_CALL ? 4 : T::WORDS + 4];   // +4: the joined-word read of the last group
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     uint32_t* wb = wordbuf[warp];
 
-    for (uint64_t tile = (uint64_t)blockIdx.x * WARPS_PER_CTA + warp; tile < n_tiles;
-         tile += (uint64_t)gridDim.x * WARPS_PER_CTA) {
+    for (uint64_t tile = (uint64_t)(blockIdx.x - first_tile_cta) * WARPS_PER_CTA + warp; tile < n_tiles;
+         tile += (uint64_t)(gridDim.x - first_tile_cta) * WARPS_PER_CTA) {
         const size_t e0 = (size_t)tile * T::ELEMS;
         const uint64_t tile_call0 = call0 + tile * T::CALLS;
 
