@@ -39,6 +39,22 @@ def sweep():
     return [(f, v, k) for f in FMT_LIST for v in VARIANT_LIST for k in K_LIST]
 
 
+# DRAM traffic of one 2^28-element bf16 launch, from the ncu capture summarised in
+# profiles/tile_kernel_round_bf16_srf_k4.txt (dram__bytes_read.sum + dram__bytes_write.sum of a 2^27-element
+# launch, scaled by the elements processed).  Valid only for the kernel sources it was taken from.
+TRAFFIC_BYTES_PER_LAUNCH = 2 * (536.895744e6 + 222.235136e6)
+TRAFFIC_KERNEL_SHA = "a8b81eeb66333071"
+
+
+def kernel_source_sha():
+    import hashlib
+    h = hashlib.sha256()
+    for name in ("fbsr_device.cuh", "fbsr_kernels.cuh"):
+        with open(os.path.join(ROOT, "paper_2504_20634_b200", "csrc", name), "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()[:16]
+
+
 def measured_peak_gbs():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     try:
@@ -211,7 +227,8 @@ def main():
     peak, peak_kind = measured_peak_gbs()
     achieved = BYTES_PER_ELEM * n_local * len(combos) / (ms_per_step * 1e-3) / 1e9
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                "traffic": None, "peak_source": peak_kind + " copy bandwidth",
+                "traffic": TRAFFIC_BYTES_PER_LAUNCH if kernel_source_sha() == TRAFFIC_KERNEL_SHA else None,
+                "peak_source": peak_kind + " copy bandwidth",
                 "kernel": "fbsr::tile_kernel<RoundOp, fmt, variant, k> (average over the 48 launches of a step)",
                 "algorithmic_bytes_per_launch": BYTES_PER_ELEM * n_local,
                 "frac_of_8TBps": achieved / 8000.0}

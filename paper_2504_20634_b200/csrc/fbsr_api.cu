@@ -234,6 +234,9 @@ int fbsr_round_host(const float* src_host, void* dst_host, size_t n, int fmt, in
     const size_t max_chunk = (size_t)1 << 26;               // keeps the first copy from delaying the first kernel
     if (chunk > max_chunk) chunk = max_chunk / tile * tile;
     if (chunk == 0) return FBSR_ERR_WORKSPACE;
+    // equal chunks (rounded up to whole tiles) instead of full chunks plus a sliver
+    const size_t n_chunks = (n + chunk - 1) / chunk;
+    chunk = ((n + n_chunks - 1) / n_chunks + tile - 1) / tile * tile;
     char* slot_in[2]; char* slot_out[2];
     const size_t in_bytes = (chunk * 4 + 255) / 256 * 256, out_bytes = (chunk * cb + 255) / 256 * 256;
     for (int i = 0; i < 2; ++i) {
