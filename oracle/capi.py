@@ -65,6 +65,8 @@ def lib():
         vp, sz, i, u64, f = ctypes.c_void_p, ctypes.c_size_t, ctypes.c_int, ctypes.c_uint64, ctypes.c_float
         L.fbsr_oracle_round.argtypes = [vp, vp, sz, i, i, i, u64, u64, f]
         L.fbsr_oracle_round_bits.argtypes = [vp, vp, sz, i, i, i, vp, f]
+        L.fbsr_oracle_round_lp.argtypes = [vp, i, vp, sz, i, i, i, u64, u64, f]
+        L.fbsr_oracle_round_lp.restype = ctypes.c_int
         L.fbsr_oracle_round_stats.argtypes = [vp, vp, sz, i, i, i, u64, u64, f, sz, vp, vp,
                                               ctypes.POINTER(OracleStats)]
         L.fbsr_oracle_sgd_update.argtypes = [vp, vp, vp, vp, sz, i, i, i, u64, u64, f, f]
@@ -151,6 +153,15 @@ def fbsr_round(src, fmt, variant, k, seed, offset=0, scale=1.0):
     dst = np.empty(src.size, dtype=CODE_DTYPE[fmt])
     _check(lib().fbsr_oracle_round(_ptr(src), _ptr(dst), src.size, FMT[fmt], VARIANT[variant], k,
                                    seed, offset, scale))
+    return dst
+
+
+def fbsr_round_lp(src_codes, src_fmt, fmt, variant, k, seed, offset=0, scale=1.0):
+    """Round an array of low-precision codes (format src_fmt) to format fmt."""
+    src = np.ascontiguousarray(src_codes, dtype=CODE_DTYPE[src_fmt])
+    dst = np.empty(src.size, dtype=CODE_DTYPE[fmt])
+    _check(lib().fbsr_oracle_round_lp(_ptr(src), FMT[src_fmt], _ptr(dst), src.size, FMT[fmt], VARIANT[variant], k,
+                                      seed, offset, scale))
     return dst
 
 

@@ -261,6 +261,21 @@ int fbsr_oracle_round_bits(const float* src, void* dst, size_t n, int fmt, int v
     return 0;
 }
 
+/* Low-precision source (the paper's own regime, Section III-E and Algorithm 1: BFloat16 or
+ * binary16 values rounded to an 8-bit format): the stored code is widened exactly by Eq. (1),
+ * scaled, and rounded like any other binary32 value.  A NaN source keeps its sign. */
+int fbsr_oracle_round_lp(const void* src, int src_fmt, void* dst, size_t n, int dst_fmt, int variant, int k,
+                         uint64_t seed, uint64_t offset, float scale)
+{
+    if (bad_args(dst_fmt, variant, k) || src_fmt < 0 || src_fmt > 3) return 1;
+    for (size_t i = 0; i < n; ++i) {
+        float y = scaled(fbsr_oracle_decode(src_fmt, load_code(src, i, src_fmt)), scale);
+        uint32_t nr = fbsr_oracle_draw(seed, offset + i, k, 0u);
+        store_code(dst, i, dst_fmt, fbsr_oracle_round_one(y, dst_fmt, variant, k, nr, 0, 0, 0));
+    }
+    return 0;
+}
+
 /* Error of one SR-rounded element in target ulps: e = up - delta~ (the
  * quantity whose mean Section III calls bias).  Group g holds elements
  * [g*group_size, (g+1)*group_size) of this call. */
