@@ -97,6 +97,16 @@ typedef struct {
 int fbsr_round(const float* src, void* dst, size_t n, int fmt, int variant, int k_bits,
                uint64_t seed, uint64_t offset, float scale, void* cuda_stream);
 
+/* fbsr_round_lp -- the paper's own regime (Section III-E, Fig. 2, Algorithm 1 "w8 <- RoundTo8(...)"):
+ * the source is already a low-precision tensor.  dst[i] = FBSR(fl32(value(src[i]) * scale)), where
+ * value() widens the stored code exactly by Eq. (1).
+ *   src      device, n codes of src_fmt (FBSR_BF16 or FBSR_FP16, uint16 each); must not overlap dst
+ *   dst      device, n codes of dst_fmt (FBSR_E4M3 or FBSR_E5M2, uint8 each)
+ * Other format pairs return FBSR_ERR_UNSUPPORTED.  The fast path needs src and dst 16-byte aligned
+ * (8-byte for dst) and `offset` on the tile grid, like fbsr_round.  A NaN source keeps its sign. */
+int fbsr_round_lp(const void* src, int src_fmt, void* dst, size_t n, int dst_fmt, int variant, int k_bits,
+                  uint64_t seed, uint64_t offset, float scale, void* cuda_stream);
+
 /* fbsr_round_bits -- the same rounding with caller-supplied random bits
  * (Section II-B: "random numbers will be supplied as a finite sequence of random
  * bits").  rand_words: device, ceil(n / dpw) words; element i uses field

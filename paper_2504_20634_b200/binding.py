@@ -40,6 +40,8 @@ def _load():
     vp, sz, i, u64, f = ctypes.c_void_p, ctypes.c_size_t, ctypes.c_int, ctypes.c_uint64, ctypes.c_float
     L.fbsr_round.argtypes = [vp, vp, sz, i, i, i, u64, u64, f, vp]
     L.fbsr_round_bits.argtypes = [vp, vp, sz, i, i, i, vp, f, vp]
+    L.fbsr_round_lp.argtypes = [vp, i, vp, sz, i, i, i, u64, u64, f, vp]
+    L.fbsr_round_lp.restype = i
     L.fbsr_stats_workspace_bytes.argtypes = []
     L.fbsr_stats_workspace_bytes.restype = sz
     L.fbsr_round_stats.argtypes = [vp, vp, sz, i, i, i, u64, u64, f, sz, vp, vp, vp, vp, sz, vp]
@@ -137,6 +139,16 @@ def fbsr_round(src, fmt, variant, k_bits, seed, offset=0, scale=1.0, out=None):
     with torch.cuda.device(src.device):
         _check(_L.fbsr_round(_dev(src, torch.float32, "src"), po, src.numel(), _fmt(fmt), _var(variant), k_bits,
                              seed, offset, scale, _stream(src)), "fbsr_round")
+    return out
+
+
+def fbsr_round_lp(src_codes, src_fmt, fmt, variant, k_bits, seed, offset=0, scale=1.0, out=None):
+    """Round a tensor of bf16/fp16 codes (uint16) to an 8-bit format; returns the uint8 codes."""
+    out, po = _out(src_codes, fmt, out)
+    with torch.cuda.device(src_codes.device):
+        _check(_L.fbsr_round_lp(_dev(src_codes, torch.uint16, "src_codes"), _fmt(src_fmt), po, src_codes.numel(),
+                                _fmt(fmt), _var(variant), k_bits, seed, offset, scale, _stream(src_codes)),
+               "fbsr_round_lp")
     return out
 
 

@@ -62,6 +62,21 @@ int fbsr_round(const float* src, void* dst, size_t n, int fmt, int variant, int 
     return finish(kRound[fmt](a));
 }
 
+int fbsr_round_lp(const void* src, int src_fmt, void* dst, size_t n, int dst_fmt, int variant, int k_bits,
+                  uint64_t seed, uint64_t offset, float scale, void* cuda_stream)
+{
+    if (bad_enum(dst_fmt, variant, k_bits) || src_fmt < 0 || src_fmt > 3) return FBSR_ERR_INVALID_ARG;
+    if (!(scale > 0.0f) || !std::isfinite(scale)) return FBSR_ERR_INVALID_ARG;
+    if ((src_fmt != FBSR_BF16 && src_fmt != FBSR_FP16) || (dst_fmt != FBSR_E4M3 && dst_fmt != FBSR_E5M2))
+        return FBSR_ERR_UNSUPPORTED;
+    if (n > 0 && (src == nullptr || dst == nullptr)) return FBSR_ERR_INVALID_ARG;
+    if (misaligned(src, 2)) return FBSR_ERR_ALIGNMENT;
+    if (n == 0) return FBSR_OK;
+    CallArgs a = base_args(OP_ROUND_LP, variant, k_bits, n, seed, offset, dst, cuda_stream);
+    a.src_lp = src; a.src_fmt = src_fmt; a.scale = scale;
+    return finish(dst_fmt == FBSR_E4M3 ? dispatch_lp_2(a) : dispatch_lp_3(a));
+}
+
 int fbsr_round_bits(const float* src, void* dst, size_t n, int fmt, int variant, int k_bits,
                     const uint32_t* rand_words, float scale, void* cuda_stream)
 {

@@ -1,6 +1,6 @@
 // Kernel instantiations and launch logic for one target format and one group of
 // operations.  Compiled once per (FBSR_FMT, FBSR_GROUP): FBSR_GROUP 0 = rounding
-// entry points, 1 = fused optimizer / accumulation entry points.
+// entry points, 1 = fused optimizer / accumulation entry points, 2 = 16-bit sources (8-bit targets only).
 #include <array>
 #include <utility>
 
@@ -11,7 +11,7 @@
 #error "compile with -DFBSR_FMT=0..3"
 #endif
 #ifndef FBSR_GROUP
-#error "compile with -DFBSR_GROUP=0|1"
+#error "compile with -DFBSR_GROUP=0|1|2"
 #endif
 
 namespace fbsr {
@@ -37,6 +37,15 @@ inline bool op_aligned(const AccumOp<FMT>& o, size_t h) { return aligned(o.u + h
 inline AccumOp<FMT> op_advance(AccumOp<FMT> o, size_t h)
 {
     o.u += h; o.w_lp = static_cast<const char*>(o.w_lp) + h * CODE_BYTES; return o;
+}
+
+template <int SRC> inline bool op_aligned(const LpSrcOp<SRC>& o, size_t h)
+{
+    return aligned(static_cast<const uint16_t*>(o.src) + h, 16);
+}
+template <int SRC> inline LpSrcOp<SRC> op_advance(LpSrcOp<SRC> o, size_t h)
+{
+    o.src = static_cast<const uint16_t*>(o.src) + h; return o;
 }
 
 struct Plan { size_t head, n_tiles, tail_begin; };
@@ -152,6 +161,14 @@ int FBSR_CAT(dispatch_round_, FBSR_FMT)(const CallArgs& a)
     }
     default: return 1;
     }
+}
+#elif FBSR_GROUP == 2
+int FBSR_CAT(dispatch_lp_, FBSR_FMT)(const CallArgs& a)
+{
+    static_assert(CODE_BYTES == 1, "16-bit sources are rounded to 8-bit targets");
+    if (a.src_fmt == BF16) return by_variant_and_k<LpSrcOp<BF16>, false>(LpSrcOp<BF16>{a.src_lp, a.scale}, a);
+    if (a.src_fmt == FP16) return by_variant_and_k<LpSrcOp<FP16>, false>(LpSrcOp<FP16>{a.src_lp, a.scale}, a);
+    return 1;
 }
 #else
 int FBSR_CAT(dispatch_optim_, FBSR_FMT)(const CallArgs& a)

@@ -6,7 +6,7 @@
 
 namespace fbsr {
 
-enum OpKind { OP_ROUND = 0, OP_ROUND_BITS, OP_ROUND_STATS, OP_SGD, OP_ADAM, OP_ACCUM };
+enum OpKind { OP_ROUND = 0, OP_ROUND_BITS, OP_ROUND_STATS, OP_SGD, OP_ADAM, OP_ACCUM, OP_ROUND_LP };
 
 // Everything an entry point hands to the per-format dispatcher.  Validated by the caller.
 struct CallArgs {
@@ -20,6 +20,8 @@ struct CallArgs {
     const float* src;
     float scale;
     const uint32_t* words;          // OP_ROUND_BITS
+    const void* src_lp;             // OP_ROUND_LP: codes of src_fmt
+    int src_fmt;
     // OP_ROUND_STATS
     size_t group_size;
     double* gsum_e;
@@ -34,10 +36,12 @@ struct CallArgs {
 
 constexpr int MAX_SLOW_GRID = 148 * 8;      // CTAs of the general kernel; also the number of partial slots
 
-// One dispatcher per (format, op group); each lives in its own translation unit.
+// One dispatcher per (format, op group); each lives in its own translation unit
+// (dispatch_lp_* exists for the 8-bit targets only).
 #define FBSR_DECLARE_DISPATCH(fmt) \
     int dispatch_round_##fmt(const CallArgs&); \
-    int dispatch_optim_##fmt(const CallArgs&);
+    int dispatch_optim_##fmt(const CallArgs&);\
+    int dispatch_lp_##fmt(const CallArgs&);
 FBSR_DECLARE_DISPATCH(0) FBSR_DECLARE_DISPATCH(1) FBSR_DECLARE_DISPATCH(2) FBSR_DECLARE_DISPATCH(3)
 #undef FBSR_DECLARE_DISPATCH
 

@@ -21,6 +21,8 @@
 // freshly updated master weight (SGD-momentum, Adam) or the widened stored
 // weight plus its update (accumulate).
 #pragma once
+#include <cuda_fp16.h>
+
 #include "fbsr_device.cuh"
 
 namespace fbsr {
@@ -148,6 +150,53 @@ struct RoundOp {
         return y != y ? __float_as_uint(x[c]) : __float_as_uint(y);   // a NaN keeps the input's sign
     }
     __device__ __forceinline__ uint32_t scalar(size_t i) const { return scaled_bits(src[i], scale); }
+};
+
+// Source already in a 16-bit format: widen exactly (Eq. (1)), then scale.
+template <int SRC>
+struct LpSrcOp {
+    static_assert(SRC == BF16 || SRC == FP16, "16-bit sources");
+    static constexpr int BATCH = ROW_BATCH, MIN_CTAS = FBSR_MIN_CTAS_ROUND;
+    const void* src;
+    float scale;
+    struct Regs { uint4 c; };
+    __device__ __forceinline__ static float widen(uint32_t code)
+    {
+        if constexpr (SRC == BF16) return __uint_as_float(code << 16);
+        else return __half2float(__ushort_as_half((unsigned short)code));
+    }
+    __device__ __forceinline__ void fetch(size_t elem, Regs& r) const
+    {
+        const uint4* p = reinterpret_cast<const uint4*>(static_cast<const uint16_t*>(src) + elem);
+        asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                     : "=r"(r.c.x), "=r"(r.c.y), "=r"(r.c.z), "=r"(r.c.w) : "l"(p));
+    }
+    __device__ __forceinline__ uint32_t code_of(const Regs& r, int c) const
+    {
+        const uint32_t w = c < 2 ? r.c.x : c < 4 ? r.c.y : c < 6 ? r.c.z : r.c.w;
+        return (c & 1) ? (w >> 16) : (w & 0xFFFFu);
+    }
+    __device__ __forceinline__ void finish(size_t, const Regs& r, float (&y)[8]) const
+    {
+        const uint32_t cw[4] = {r.c.x, r.c.y, r.c.z, r.c.w};
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+            float v;
+            if constexpr (SRC == BF16) v = __uint_as_float((c & 1) ? (cw[c >> 1] & 0xFFFF0000u) : (cw[c >> 1] << 16));
+            else v = widen((c & 1) ? (cw[c >> 1] >> 16) : (cw[c >> 1] & 0xFFFFu));
+            y[c] = __fmul_rn(v, scale);
+        }
+    }
+    __device__ __forceinline__ uint32_t exact_bits(const Regs& r, int c, float y) const
+    {
+        // a NaN keeps the sign of the stored code
+        return y != y ? __float_as_uint(decode_element<SRC>(code_of(r, c))) : __float_as_uint(y);
+    }
+    __device__ __forceinline__ uint32_t scalar(size_t i) const
+    {
+        const float v = decode_element<SRC>(static_cast<const uint16_t*>(src)[i]);
+        return scaled_bits(v, scale);
+    }
 };
 
 // m' = fma(mu, m, g);  w' = fma(-lr, m', w)

@@ -28,6 +28,25 @@ def bias_grid(cell_centred=True, points=1024, repeats=5000, device="cpu"):
     return x.to(torch.float32).repeat_interleave(repeats).to(device)
 
 
+def fig2_grid(repeats=100_000, device="cpu"):
+    """Fig. 2 shape: every BFloat16 value of the binade [1, 2) (128 codes), each repeated `repeats`
+    times contiguously, as uint16 codes."""
+    codes = torch.arange(0x3F80, 0x4000, dtype=torch.int32).to(torch.uint16)
+    return codes.repeat_interleave(repeats).to(device)
+
+
+def lp_sweep(n, src_fmt="bf16", seed=1234, device="cpu"):
+    """The bandwidth-sweep distribution narrowed to a 16-bit source format (torch's nearest-even
+    cast), as uint16 codes; magnitudes span 2^-12..2^12 so that both 8-bit targets see their normal,
+    subnormal and saturating ranges."""
+    g = _gen(seed, device)
+    z = torch.randn(n, generator=g, device=device, dtype=torch.float32)
+    e = torch.rand(n, generator=g, device=device, dtype=torch.float32) * 24.0 - 12.0
+    x = z * torch.exp2(e)
+    dt = torch.bfloat16 if src_fmt == "bf16" else torch.float16
+    return x.to(dt).view(torch.uint16)
+
+
 def bandwidth_sweep(n, seed=1234, device="cpu"):
     """z ~ N(0, 1) times a log-uniform factor 2^U(-20, 20), per element."""
     g = _gen(seed, device)
