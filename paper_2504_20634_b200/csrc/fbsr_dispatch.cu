@@ -24,17 +24,17 @@ inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_
 
 // Host view of an Op: which pointers the tiled kernel reads with 256-bit accesses, and
 // the same Op with every pointer moved forward by h elements.
-inline bool op_aligned(const RoundOp& o, size_t h) { return aligned(o.src + h, 32); }
-inline RoundOp op_advance(RoundOp o, size_t h) { o.src += h; return o; }
-inline bool op_aligned(const SgdOp& o, size_t h) { return aligned(o.w + h, 32) && aligned(o.g + h, 32) && aligned(o.m + h, 32); }
-inline SgdOp op_advance(SgdOp o, size_t h) { o.w += h; o.g += h; o.m += h; return o; }
-inline bool op_aligned(const AdamOp& o, size_t h)
+[[maybe_unused]] inline bool op_aligned(const RoundOp& o, size_t h) { return aligned(o.src + h, 32); }
+[[maybe_unused]] inline RoundOp op_advance(RoundOp o, size_t h) { o.src += h; return o; }
+[[maybe_unused]] inline bool op_aligned(const SgdOp& o, size_t h) { return aligned(o.w + h, 32) && aligned(o.g + h, 32) && aligned(o.m + h, 32); }
+[[maybe_unused]] inline SgdOp op_advance(SgdOp o, size_t h) { o.w += h; o.g += h; o.m += h; return o; }
+[[maybe_unused]] inline bool op_aligned(const AdamOp& o, size_t h)
 {
     return aligned(o.w + h, 32) && aligned(o.g + h, 32) && aligned(o.m + h, 32) && aligned(o.v + h, 32);
 }
-inline AdamOp op_advance(AdamOp o, size_t h) { o.w += h; o.g += h; o.m += h; o.v += h; return o; }
-inline bool op_aligned(const AccumOp<FMT>& o, size_t h) { return aligned(o.u + h, 32); }
-inline AccumOp<FMT> op_advance(AccumOp<FMT> o, size_t h)
+[[maybe_unused]] inline AdamOp op_advance(AdamOp o, size_t h) { o.w += h; o.g += h; o.m += h; o.v += h; return o; }
+[[maybe_unused]] inline bool op_aligned(const AccumOp<FMT>& o, size_t h) { return aligned(o.u + h, 32); }
+[[maybe_unused]] inline AccumOp<FMT> op_advance(AccumOp<FMT> o, size_t h)
 {
     o.u += h; o.w_lp = static_cast<const char*>(o.w_lp) + h * CODE_BYTES; return o;
 }

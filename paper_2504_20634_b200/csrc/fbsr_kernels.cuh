@@ -398,7 +398,6 @@ tile_kernel(const Op op, void* __restrict__ dst, const uint64_t n_tiles, const u
             __syncwarp();
         }
 
-#pragma unroll
         // rows are taken in equal batches of at most Op::BATCH (5 rows: 3 + 2, not 4 + 1)
         constexpr int N_BATCHES = (T::ROWS + Op::BATCH - 1) / Op::BATCH;
         constexpr int BATCH = (T::ROWS + N_BATCHES - 1) / N_BATCHES;

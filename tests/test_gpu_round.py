@@ -35,6 +35,24 @@ def test_every_format_variant_and_k(fmt, variant):
         assert gu.canaries_intact(raw, n, fbsr.CODE_DTYPE[fmt])
 
 
+@pytest.mark.parametrize("fmt", FMTS)
+def test_whole_binary32_exponent_range_and_extreme_scales(fmt):
+    """Inputs drawn uniformly over every binary32 bit pattern (all exponents, subnormals, NaNs, infinities)
+    and scales from 2^-100 to 2^100: the rescaling and the special-value detection of the fast rows must
+    agree with the oracle everywhere, including where the scaled value under- or overflows binary32."""
+    rng = np.random.default_rng(FMTS.index(fmt) + 70)
+    n = 40 * 1024 + 77
+    pats = rng.integers(0, 1 << 32, size=n, dtype=np.uint64).astype(np.uint32)
+    x = pats.view(np.float32)
+    xd = torch.from_numpy(x).cuda()
+    for k in (1, 3, 5, 8, 11, 12, 13, 14, 16):
+        for variant in VARIANTS:
+            for scale in (1.0, 2.0 ** -100, 2.0 ** 100, 3.0e-39, 1.0e30, 0.3333333):
+                got = fbsr.fbsr_round(xd, fmt, variant, k, seed=k, offset=0, scale=scale)
+                expect = capi.fbsr_round(x, fmt, variant, k, seed=k, offset=0, scale=scale)
+                gu.assert_codes_equal(got, expect, "%s %s k=%d scale=%g" % (fmt, variant, k, scale))
+
+
 @pytest.mark.parametrize("fmt", ["bf16", "e4m3"])
 def test_small_and_ragged_sizes(fmt):
     for k in (1, 2, 3, 6, 8, 13, 16):
