@@ -16,7 +16,7 @@ _LIB = os.path.join(_HERE, "libfbsr_oracle.so")
 _CFLAGS = ["-O2", "-std=gnu11", "-ffp-contract=off", "-fno-fast-math", "-shared", "-fPIC"]
 
 FMT = {"bf16": 0, "fp16": 1, "e4m3": 2, "e5m2": 3}
-VARIANT = {"srff": 0, "srf": 1, "src": 2}
+VARIANT = {"srff": 0, "srf": 1, "src": 2, "rtne": 3, "rta": 4, "rto": 5}
 CODE_DTYPE = {"bf16": np.uint16, "fp16": np.uint16, "e4m3": np.uint8, "e5m2": np.uint8}
 
 
@@ -74,6 +74,8 @@ def lib():
         L.fbsr_oracle_adam_coefficients.argtypes = [f, f, f, i, ctypes.POINTER(ctypes.c_float)]
         L.fbsr_oracle_adam_coefficients.restype = None
         L.fbsr_oracle_accumulate.argtypes = [vp, vp, sz, i, i, i, u64, u64]
+        L.fbsr_oracle_qat_update.argtypes = [vp, vp, sz, i, i, i, i, u64, u64]
+        L.fbsr_oracle_qat_update.restype = ctypes.c_int
         for name in ("round", "round_bits", "round_stats", "sgd_update", "adam_update", "accumulate"):
             getattr(L, "fbsr_oracle_" + name).restype = ctypes.c_int
         _lib = L
@@ -220,3 +222,12 @@ def accumulate(w_lp, update, fmt, variant, k, seed, offset=0):
     _check(lib().fbsr_oracle_accumulate(_ptr(w_lp), _ptr(update), w_lp.size, FMT[fmt], VARIANT[variant], k,
                                         seed, offset))
     return w_lp
+
+
+def qat_update(w8, u16, w_fmt, u_fmt, variant, k, seed, offset=0):
+    """In place on w8 (8-bit codes): w8 <- FBSR(RTNE16(value(w8) + value(u16)))."""
+    assert w8.dtype == np.uint8 and w8.flags.c_contiguous
+    u16 = np.ascontiguousarray(u16, dtype=np.uint16)
+    _check(lib().fbsr_oracle_qat_update(_ptr(w8), _ptr(u16), w8.size, FMT[w_fmt], FMT[u_fmt], VARIANT[variant], k,
+                                        seed, offset))
+    return w8

@@ -16,6 +16,8 @@
  *                            R_SRF (d, n) = d + (n + 1/2) 2^-N >= 1
  *   Section III-F, Eq. (8)   R_SRC(d, n) = R_SRFF(Round(d 2^N) 2^-N, n), Round =
  *                            nearest, ties to even
+ *   Section II-A, Eq. (4)    deterministic modes (no draw): R_TA(d) = d >= 1/2;
+ *                            R_TNE = d > 1/2 or (d = 1/2 and floor(sigma~)+1 even); ties-to-odd likewise
  *
  * The input is binary32, so delta~ is the rational r / 2^s with r, s integers.
  * Each predicate is evaluated exactly by clearing denominators in 128-bit
@@ -44,7 +46,7 @@
 typedef unsigned __int128 u128;
 
 enum { FMT_BF16 = 0, FMT_FP16 = 1, FMT_E4M3 = 2, FMT_E5M2 = 3 };
-enum { VAR_SRFF = 0, VAR_SRF = 1, VAR_SRC = 2 };
+enum { VAR_SRFF = 0, VAR_SRF = 1, VAR_SRC = 2, VAR_RTNE = 3, VAR_RTA = 4, VAR_RTO = 5 };
 enum { KIND_FINITE = 0, KIND_NAN = 1, KIND_INF = 2, KIND_SAT = 3 };
 
 typedef struct {
@@ -173,7 +175,8 @@ uint32_t fbsr_oracle_round_one(float y, int fmt, int variant, int N, uint32_t n,
         uint64_t fl, r;
         if (s >= 64) {
             /* m < 2^24 so delta~ < 2^-40: with N <= 16 no predicate can hold
-               (delta~ + (n + 1/2) 2^-N <= 2^-40 + 1 - 2^-17 < 1; Round(delta~ 2^N) = 0). */
+               (delta~ + (n + 1/2) 2^-N <= 2^-40 + 1 - 2^-17 < 1; Round(delta~ 2^N) = 0;
+               delta~ < 1/2 for the deterministic modes). */
             fl = 0; r = m; up = 0;
             delta = ldexp((double)m, -s);
         } else {
@@ -184,6 +187,12 @@ uint32_t fbsr_oracle_round_one(float y, int fmt, int variant, int N, uint32_t n,
             if (variant == VAR_SRFF) {
                 /* r/2^s + n/2^N >= 1   <=>   r 2^N + n 2^s >= 2^(s+N) */
                 up = ((u128)r << N) + ((u128)n << s) >= (one << (s + N));
+            } else if (variant == VAR_RTA) {
+                up = ((u128)r << 1) >= (one << s);                                   /* delta >= 1/2 */
+            } else if (variant == VAR_RTNE || variant == VAR_RTO) {
+                u128 twice = (u128)r << 1, den = one << s;
+                int next_is_even = ((fl + 1) & 1u) == 0;
+                up = twice > den || (twice == den && (variant == VAR_RTNE ? next_is_even : !next_is_even));
             } else if (variant == VAR_SRF) {
                 /* r/2^s + (2n+1)/2^(N+1) >= 1 */
                 up = ((u128)r << (N + 1)) + ((u128)(2u * n + 1u) << s) >= (one << (s + N + 1));
@@ -233,7 +242,7 @@ static float arith_result(float y) { return isnan(y) ? NAN : y; }
 
 static int bad_args(int fmt, int variant, int k)
 {
-    return fmt < 0 || fmt > 3 || variant < 0 || variant > 2 || k < 1 || k > 16;
+    return fmt < 0 || fmt > 3 || variant < 0 || variant > 5 || k < 1 || k > 16;
 }
 
 /* ------------------------------------------------------------ array forms */
@@ -367,6 +376,26 @@ int fbsr_oracle_adam_update(float* w, const float* g, float* m, float* v, void* 
         m[i] = m2; v[i] = v2; w[i] = w2;
         uint32_t nr = fbsr_oracle_draw(seed, offset + i, k, 0u);
         store_code(dst, i, fmt, fbsr_oracle_round_one(arith_result(w2), fmt, variant, k, nr, 0, 0, 0));
+    }
+    return 0;
+}
+
+/* Algorithm 1, last line, with the sum formed in the 16-bit format as the algorithm states
+ * ("w8 <- RoundTo8(w16 + u16)"): w16 = value(w8) exactly; s = fl32(w16 + u16) rounded to the 16-bit
+ * format with ties to even (saturating like every other rounding here); w8' = FBSR(s).  Forming the
+ * 16-bit sum by way of one binary32 addition is this library's definition. */
+int fbsr_oracle_qat_update(void* w8, const void* u16, size_t n, int w_fmt, int u_fmt, int variant, int k,
+                           uint64_t seed, uint64_t offset)
+{
+    if (bad_args(w_fmt, variant, k) || u_fmt < 0 || u_fmt > 1 || w_fmt < 2) return 1;
+    for (size_t i = 0; i < n; ++i) {
+        float wv = fbsr_oracle_decode(w_fmt, load_code(w8, i, w_fmt));
+        float uv = fbsr_oracle_decode(u_fmt, load_code(u16, i, u_fmt));
+        float s32 = arith_result(wv + uv);
+        uint32_t s16 = fbsr_oracle_round_one(s32, u_fmt, VAR_RTNE, 1, 0u, 0, 0, 0);
+        float y = arith_result(fbsr_oracle_decode(u_fmt, s16));
+        uint32_t nr = fbsr_oracle_draw(seed, offset + i, k, 0u);
+        store_code(w8, i, w_fmt, fbsr_oracle_round_one(y, w_fmt, variant, k, nr, 0, 0, 0));
     }
     return 0;
 }

@@ -44,7 +44,8 @@ FORMATS = {
 }
 FORMAT_IDS = {"bf16": 0, "fp16": 1, "e4m3": 2, "e5m2": 3}
 VARIANTS = ("srff", "srf", "src")
-VARIANT_IDS = {"srff": 0, "srf": 1, "src": 2}
+DETERMINISTIC = ("rtne", "rta", "rto")          # Section II-A: ties to even, ties away, ties to odd
+VARIANT_IDS = {"srff": 0, "srf": 1, "src": 2, "rtne": 3, "rta": 4, "rto": 5}
 
 
 def pow2(e):
@@ -172,6 +173,23 @@ def r_src(delta, n, N):
     return r_srff(round_nearest_even(delta * pow2(N)) * pow2(-N), n, N)
 
 
+def r_ta(delta):
+    """R_TA(delta) = delta >= 0.5   (Section II-A, Eq. (4))."""
+    return delta >= Fraction(1, 2)
+
+
+def r_tne(sig, delta):
+    """R_TNE(sigma~, delta) = delta > 0.5 or (delta = 0.5 and IsEven(floor(sigma~) + 1))   (Section II-A)."""
+    fl = sig.numerator // sig.denominator
+    return delta > Fraction(1, 2) or (delta == Fraction(1, 2) and (fl + 1) % 2 == 0)
+
+
+def r_tno(sig, delta):
+    """Ties to odd, the analogue the paper mentions next to R_TNE."""
+    fl = sig.numerator // sig.denominator
+    return delta > Fraction(1, 2) or (delta == Fraction(1, 2) and (fl + 1) % 2 == 1)
+
+
 PREDICATES = {"srff": r_srff, "srf": r_srf, "src": r_src}
 
 
@@ -183,12 +201,19 @@ def round_positive(xt, fmt, variant, n, N):
     """
     f = FORMATS[fmt]
     P, B = f["P"], f["B"]
-    assert xt > 0 and 0 <= n < (1 << N)
+    assert xt > 0 and (variant in DETERMINISTIC or 0 <= n < (1 << N))
     e = max(floor_log2(xt), 1 - B)                     # Eq. (2)
     sig = xt * pow2(-e) * pow2(P - 1)                  # Eq. (3)
     fl = sig.numerator // sig.denominator
     delta = sig - fl
-    up = 1 if PREDICATES[variant](delta, n, N) else 0
+    if variant == "rta":
+        up = 1 if r_ta(delta) else 0
+    elif variant == "rtne":
+        up = 1 if r_tne(sig, delta) else 0
+    elif variant == "rto":
+        up = 1 if r_tno(sig, delta) else 0
+    else:
+        up = 1 if PREDICATES[variant](delta, n, N) else 0
     sigma = fl + up                                    # Eq. (5)
     rounded_value = sigma * pow2(e - (P - 1))
     if sigma == (1 << P):                              # exponent increment
