@@ -66,8 +66,13 @@ typedef enum {
     FBSR_E5M2 = 3  /* ( 8,  3,  15; 57344) */
 } fbsr_fmt;
 
-/* Round-up predicates, Section II-B and Eq. (8). */
-typedef enum { FBSR_SRFF = 0, FBSR_SRF = 1, FBSR_SRC = 2 } fbsr_variant;
+/* Round-up predicates: the few-bit stochastic ones of Section II-B and Eq. (8), and the deterministic
+ * ones of Section II-A (ties to even, ties away from zero (Eq. (4)), ties to odd), which use no draw:
+ * for those k_bits, seed and offset are ignored (k_bits must still be in 1..16). */
+typedef enum {
+    FBSR_SRFF = 0, FBSR_SRF = 1, FBSR_SRC = 2,
+    FBSR_RTNE = 3, FBSR_RTA = 4, FBSR_RTO = 5
+} fbsr_variant;
 
 /* Error statistics over the SR-rounded elements of one call.  e = up - delta~
  * is the rounding error of the magnitude in target ulps, the quantity whose
@@ -190,6 +195,14 @@ int fbsr_adam_update(float* master_w, const float* grad, float* m, float* v, voi
  * formed in binary32:  w_lp[i] = FBSR(fl32(value(w_lp[i]) + update[i])), in place.
  * A NaN sum is written as the positive quiet NaN. */
 int fbsr_accumulate(void* w_lp, const float* update, size_t n, int fmt, int variant, int k_bits,
+                    uint64_t seed, uint64_t offset, void* cuda_stream);
+
+/* fbsr_qat_update -- Algorithm 1, last line, with the sum formed in the 16-bit format as written there:
+ *     w16 = value(w8);  s = RTNE_16(fl32(w16 + u16));  w8 = FBSR(s)          (in place on w8)
+ *   w8       device, n codes of w_fmt (FBSR_E4M3 or FBSR_E5M2), read and overwritten
+ *   update16 device, n codes of u_fmt (FBSR_BF16 or FBSR_FP16): the update computed in the 16-bit format
+ * RTNE_16 rounds to u_fmt with ties to even (saturating); a NaN sum is written as the positive NaN. */
+int fbsr_qat_update(void* w8, const void* update16, size_t n, int w_fmt, int u_fmt, int variant, int k_bits,
                     uint64_t seed, uint64_t offset, void* cuda_stream);
 
 /* fbsr_round_host -- fbsr_round for HOST buffers (pinned memory gives overlap):

@@ -14,7 +14,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_HERE, "libfbsr.so")
 
 FMT = {"bf16": 0, "fp16": 1, "e4m3": 2, "e5m2": 3}
-VARIANT = {"srff": 0, "srf": 1, "src": 2}
+VARIANT = {"srff": 0, "srf": 1, "src": 2, "rtne": 3, "rta": 4, "rto": 5}
 CODE_DTYPE = {"bf16": torch.uint16, "fp16": torch.uint16, "e4m3": torch.uint8, "e5m2": torch.uint8}
 VIEW_DTYPE = {"bf16": torch.bfloat16, "fp16": torch.float16, "e4m3": torch.float8_e4m3fn,
               "e5m2": torch.float8_e5m2}
@@ -50,6 +50,8 @@ def _load():
     L.fbsr_sgd_update.argtypes = [vp, vp, vp, vp, sz, i, i, i, u64, u64, f, f, vp]
     L.fbsr_adam_update.argtypes = [vp, vp, vp, vp, vp, sz, i, i, i, u64, u64, f, f, f, f, i, vp]
     L.fbsr_accumulate.argtypes = [vp, vp, sz, i, i, i, u64, u64, vp]
+    L.fbsr_qat_update.argtypes = [vp, vp, sz, i, i, i, i, u64, u64, vp]
+    L.fbsr_qat_update.restype = i
     L.fbsr_round_host_min_workspace.argtypes = []
     L.fbsr_round_host_min_workspace.restype = sz
     L.fbsr_round_host.argtypes = [vp, vp, sz, i, i, i, u64, u64, f, vp, sz, vp]
@@ -233,6 +235,15 @@ def fbsr_accumulate(w_lp, update, fmt, variant, k_bits, seed, offset=0):
                                   w_lp.numel(), _fmt(fmt), _var(variant), k_bits, seed, offset, _stream(w_lp)),
                "fbsr_accumulate")
     return w_lp
+
+
+def fbsr_qat_update(w8, update16, w_fmt, u_fmt, variant, k_bits, seed, offset=0):
+    """In place on w8 (uint8 codes): w8 <- FBSR(RTNE_16(value(w8) + value(update16)))."""
+    with torch.cuda.device(w8.device):
+        _check(_L.fbsr_qat_update(_dev(w8, torch.uint8, "w8"), _dev(update16, torch.uint16, "update16"), w8.numel(),
+                                  _fmt(w_fmt), _fmt(u_fmt), _var(variant), k_bits, seed, offset, _stream(w8)),
+               "fbsr_qat_update")
+    return w8
 
 
 def fbsr_round_host(src_host, dst_host, fmt, variant, k_bits, seed, offset, scale, workspace):

@@ -18,7 +18,7 @@ typedef int (*dispatch_fn)(const CallArgs&);
 const dispatch_fn kRound[4] = {dispatch_round_0, dispatch_round_1, dispatch_round_2, dispatch_round_3};
 const dispatch_fn kOptim[4] = {dispatch_optim_0, dispatch_optim_1, dispatch_optim_2, dispatch_optim_3};
 
-inline bool bad_enum(int fmt, int variant, int k) { return fmt < 0 || fmt > 3 || variant < 0 || variant > 2 || k < 1 || k > 16; }
+inline bool bad_enum(int fmt, int variant, int k) { return fmt < 0 || fmt > 3 || variant < 0 || variant > 5 || k < 1 || k > 16; }
 inline size_t code_bytes(int fmt) { return fmt <= 1 ? 2 : 1; }
 inline bool misaligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) != 0; }
 
@@ -200,6 +200,19 @@ int fbsr_accumulate(void* w_lp, const float* update, size_t n, int fmt, int vari
     CallArgs a = base_args(OP_ACCUM, variant, k_bits, n, seed, offset, w_lp, cuda_stream);
     a.src = update;
     return finish(kOptim[fmt](a));
+}
+
+int fbsr_qat_update(void* w8, const void* update16, size_t n, int w_fmt, int u_fmt, int variant, int k_bits,
+                    uint64_t seed, uint64_t offset, void* cuda_stream)
+{
+    if (bad_enum(w_fmt, variant, k_bits) || u_fmt < 0 || u_fmt > 3) return FBSR_ERR_INVALID_ARG;
+    if ((w_fmt != FBSR_E4M3 && w_fmt != FBSR_E5M2) || (u_fmt != FBSR_BF16 && u_fmt != FBSR_FP16)) return FBSR_ERR_UNSUPPORTED;
+    if (n > 0 && (!w8 || !update16)) return FBSR_ERR_INVALID_ARG;
+    if (misaligned(update16, 2)) return FBSR_ERR_ALIGNMENT;
+    if (n == 0) return FBSR_OK;
+    CallArgs a = base_args(OP_QAT, variant, k_bits, n, seed, offset, w8, cuda_stream);
+    a.src_lp = update16; a.src_fmt = u_fmt;
+    return finish(w_fmt == FBSR_E4M3 ? dispatch_lp_2(a) : dispatch_lp_3(a));
 }
 
 size_t fbsr_tile_elements(int k_bits)

@@ -19,7 +19,7 @@
 namespace fbsr {
 
 enum { BF16 = 0, FP16 = 1, E4M3 = 2, E5M2 = 3 };
-enum { SRFF = 0, SRF = 1, SRC = 2 };
+enum { SRFF = 0, SRF = 1, SRC = 2, RTNE = 3, RTA = 4, RTO = 5 };    // 3..5: Section II-A, no draw
 
 template <int FMT> struct Format;
 template <> struct Format<BF16> {
@@ -98,7 +98,10 @@ __device__ __forceinline__ uint32_t round_core(uint32_t ybits, uint32_t n, const
         // bfloat16 shares binary32's exponent range: sh is always 16 and the
         // whole of Eq. (2)-(5) is one addition on the magnitude pattern.
         uint32_t t;
-        if (VAR == SRFF || N == 16) {
+        if (VAR >= RTNE) {
+            const uint32_t floor_lsb = (mag >> 16) & 1u;
+            t = mag + (VAR == RTA ? 0x8000u : 0x7FFFu + (VAR == RTNE ? floor_lsb : floor_lsb ^ 1u));
+        } else if (VAR == SRFF || N == 16) {
             t = mag + (n << (16 - N));
         } else if (VAR == SRF) {
             t = mag + (((n << 1) | 1u) << (15 - N));
@@ -116,7 +119,12 @@ __device__ __forceinline__ uint32_t round_core(uint32_t ybits, uint32_t n, const
         const int sh = (24 - P) + (te - eb);                 // excess bits, >= 24 - P >= 13
         const uint32_t m6 = m << 6;                          // 6 guard positions keep every shift >= 0
         uint32_t sig;
-        if (VAR == SRFF) {
+        if (VAR >= RTNE) {
+            const int sa = min(sh + 6, 31);                  // >= 19
+            const uint32_t floor_lsb = (m6 >> sa) & 1u;
+            const uint32_t inc = VAR == RTA ? (1u << (sa - 1)) : ((1u << (sa - 1)) - 1u) + (VAR == RTNE ? floor_lsb : floor_lsb ^ 1u);
+            sig = (m6 + inc) >> sa;
+        } else if (VAR == SRFF) {
             const int sa = min(sh - N + 6, 31);
             sig = ((m6 >> sa) + n) >> N;
         } else if (VAR == SRF) {
@@ -155,7 +163,7 @@ template <int K> struct Draws8 {
     static constexpr bool POW2 = (DPW & (DPW - 1)) == 0;
     static constexpr int G = POW2 ? (DPW >= 8 ? 8 : DPW) : (4 * K <= 32 ? 4 : 2);
     static constexpr uint32_t MASK = (1u << K) - 1u;
-    uint32_t u[8 / G];
+    uint32_t u[8 / G] = {};
 
     // Field of element c moved so that its lowest bit lands on bit POS (0 <= POS, POS + K <= 32).
     template <int POS>
@@ -240,8 +248,9 @@ template <int FMT, int VAR, int N> struct FastRow {
     using F = Format<FMT>;
     static constexpr int SH0 = 24 - F::P;
     static constexpr bool ALL_BITS = (N == SH0);             // then every variant is exact SR
+    static constexpr bool deterministic = VAR >= RTNE;
     static constexpr bool one_regime =
-        FMT == BF16 ? true
+        FMT == BF16 || deterministic ? true
                     : (VAR == SRFF ? N <= SH0 : VAR == SRF ? N <= SH0 - 1 : N <= SH0 - 2);
 };
 
@@ -251,8 +260,8 @@ __device__ __forceinline__ bool round_row_fast(const float (&y)[8], const Draws8
     using F = Format<FMT>;
     using R = FastRow<FMT, VAR, N>;
     constexpr int SH0 = R::SH0;
-    constexpr int EFF = (R::ALL_BITS || (FMT == BF16 && N == 16)) ? SRFF : VAR;
-    constexpr int POS = SH0 - N;                              // where the draw is added
+    constexpr int EFF = R::deterministic ? VAR : (R::ALL_BITS || (FMT == BF16 && N == 16)) ? SRFF : VAR;
+    constexpr int POS = R::deterministic ? SH0 : SH0 - N;     // where the draw (or the half step) is added
     float flag = 0.0f;
     if constexpr (!R::one_regime) {
         static_assert(FMT != BF16 && N >= SH0 - 1, "two-regime form is for draws about as wide as the excess bits");
@@ -291,14 +300,19 @@ __device__ __forceinline__ bool round_row_fast(const float (&y)[8], const Draws8
         } else {
             const float rescale = __uint_as_float((uint32_t)(128 - F::EMINB) << 23);   // 2^(1 - EMINB)
             u = __float_as_uint(__fmul_rz(fabsf(y[c]), rescale));
-            if constexpr (EFF == SRC) {
+            if constexpr (EFF == SRC || EFF == RTNE || EFF == RTO) {
                 const uint32_t up = __float_as_uint(__fmul_ru(fabsf(y[c]), rescale));
                 u |= (u ^ up) & 1u;                           // sticky: round to odd
             }
             flag = __fmaf_rn(y[c], 0.0f, flag);               // NaN iff y is Inf or NaN
         }
         uint32_t sum;
-        if constexpr (EFF == SRFF) {
+        if constexpr (EFF == RTA) {
+            sum = u + (1u << (POS - 1));                      // ties away: add half a step
+        } else if constexpr (EFF == RTNE || EFF == RTO) {
+            const uint32_t floor_lsb = (u >> POS) & 1u;
+            sum = u + ((1u << (POS - 1)) - 1u) + (EFF == RTNE ? floor_lsb : floor_lsb ^ 1u);
+        } else if constexpr (EFF == SRFF) {
             sum = d.template add_at<POS>(c, u);
         } else if constexpr (EFF == SRF) {
             sum = d.template add_at<POS>(c, u + (1u << (POS - 1)));

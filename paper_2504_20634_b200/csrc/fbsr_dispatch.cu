@@ -39,6 +39,14 @@ inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_
     o.u += h; o.w_lp = static_cast<const char*>(o.w_lp) + h * CODE_BYTES; return o;
 }
 
+template <int UF> inline bool op_aligned(const QatOp<FMT == E4M3 || FMT == E5M2 ? FMT : E4M3, UF>& o, size_t h)
+{
+    return aligned(static_cast<const uint16_t*>(o.u16) + h, 16);      // w8 is checked as dst
+}
+template <int UF> inline QatOp<FMT == E4M3 || FMT == E5M2 ? FMT : E4M3, UF> op_advance(QatOp<FMT == E4M3 || FMT == E5M2 ? FMT : E4M3, UF> o, size_t h)
+{
+    o.w8 = static_cast<const uint8_t*>(o.w8) + h; o.u16 = static_cast<const uint16_t*>(o.u16) + h; return o;
+}
 template <int SRC> inline bool op_aligned(const LpSrcOp<SRC>& o, size_t h)
 {
     return aligned(static_cast<const uint16_t*>(o.src) + h, 16);
@@ -135,6 +143,10 @@ int by_variant_and_k(const Op& op, const CallArgs& a)
     using Seq = std::make_integer_sequence<int, 16>;
     static constexpr std::array<RunFn<Op, BITS>, 16> table[3] = {
         row_of<Op, BITS, SRFF>(Seq{}), row_of<Op, BITS, SRF>(Seq{}), row_of<Op, BITS, SRC>(Seq{})};
+    // the deterministic modes use no draws: one instantiation each, on the 1024-element tile of k = 16
+    if (a.variant == RTNE) return run<Op, RTNE, 16, false>(op, a);
+    if (a.variant == RTA) return run<Op, RTA, 16, false>(op, a);
+    if (a.variant == RTO) return run<Op, RTO, 16, false>(op, a);
     return table[a.variant][a.k - 1](op, a);
 }
 
@@ -166,6 +178,11 @@ int FBSR_CAT(dispatch_round_, FBSR_FMT)(const CallArgs& a)
 int FBSR_CAT(dispatch_lp_, FBSR_FMT)(const CallArgs& a)
 {
     static_assert(CODE_BYTES == 1, "16-bit sources are rounded to 8-bit targets");
+    if (a.op == OP_QAT) {
+        if (a.src_fmt == BF16) return by_variant_and_k<QatOp<FMT, BF16>, false>(QatOp<FMT, BF16>{a.dst, a.src_lp}, a);
+        if (a.src_fmt == FP16) return by_variant_and_k<QatOp<FMT, FP16>, false>(QatOp<FMT, FP16>{a.dst, a.src_lp}, a);
+        return 1;
+    }
     if (a.src_fmt == BF16) return by_variant_and_k<LpSrcOp<BF16>, false>(LpSrcOp<BF16>{a.src_lp, a.scale}, a);
     if (a.src_fmt == FP16) return by_variant_and_k<LpSrcOp<FP16>, false>(LpSrcOp<FP16>{a.src_lp, a.scale}, a);
     return 1;

@@ -6,7 +6,7 @@
 
 namespace fbsr {
 
-enum OpKind { OP_ROUND = 0, OP_ROUND_BITS, OP_ROUND_STATS, OP_SGD, OP_ADAM, OP_ACCUM, OP_ROUND_LP };
+enum OpKind { OP_ROUND = 0, OP_ROUND_BITS, OP_ROUND_STATS, OP_SGD, OP_ADAM, OP_ACCUM, OP_ROUND_LP, OP_QAT };
 
 // Everything an entry point hands to the per-format dispatcher.  Validated by the caller.
 struct CallArgs {
@@ -20,7 +20,7 @@ struct CallArgs {
     const float* src;
     float scale;
     const uint32_t* words;          // OP_ROUND_BITS
-    const void* src_lp;             // OP_ROUND_LP: codes of src_fmt
+    const void* src_lp;             // OP_ROUND_LP: codes of src_fmt; OP_QAT: the 16-bit updates
     int src_fmt;
     // OP_ROUND_STATS
     size_t group_size;

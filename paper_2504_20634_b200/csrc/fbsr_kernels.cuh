@@ -21,6 +21,7 @@
 // freshly updated master weight (SGD-momentum, Adam) or the widened stored
 // weight plus its update (accumulate).
 #pragma once
+#include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
 #include "fbsr_device.cuh"
@@ -307,6 +308,49 @@ struct AccumOp {
     }
 };
 
+// Algorithm 1, last line: w16 = value(w8); s = RTNE_16(fl32(w16 + u16)); the caller of finish() rounds s to 8 bits.
+template <int WF, int UF>
+struct QatOp {
+    static_assert((WF == E4M3 || WF == E5M2) && (UF == BF16 || UF == FP16), "8-bit weights, 16-bit updates");
+    static constexpr int BATCH = ROW_BATCH, MIN_CTAS = FBSR_MIN_CTAS_ROUND;
+    const void* w8; const void* u16;
+    struct Regs { uint2 w; uint4 u; };
+    __device__ __forceinline__ static float sum16(uint32_t wcode, uint32_t ucode)
+    {
+        const float wv = decode_element<WF>(wcode);
+        const float uv = UF == BF16 ? __uint_as_float(ucode << 16) : __half2float(__ushort_as_half((unsigned short)ucode));
+        float s = __fadd_rn(wv, uv);
+        // round to the 16-bit format, ties to even; a finite sum beyond its largest value saturates
+        const float m16 = __uint_as_float(Format<UF>::MAXBITS);
+        const float a = fabsf(s);
+        if (a > m16 && a < __uint_as_float(0x7F800000u)) s = copysignf(m16, s);
+        if constexpr (UF == BF16) return __bfloat162float(__float2bfloat16_rn(s));
+        else return __half2float(__float2half_rn(s));
+    }
+    __device__ __forceinline__ void fetch(size_t elem, Regs& r) const
+    {
+        r.w = *reinterpret_cast<const uint2*>(static_cast<const uint8_t*>(w8) + elem);
+        const uint4* p = reinterpret_cast<const uint4*>(static_cast<const uint16_t*>(u16) + elem);
+        asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                     : "=r"(r.u.x), "=r"(r.u.y), "=r"(r.u.z), "=r"(r.u.w) : "l"(p));
+    }
+    __device__ __forceinline__ void finish(size_t, const Regs& r, float (&y)[8]) const
+    {
+        const uint32_t uw[4] = {r.u.x, r.u.y, r.u.z, r.u.w};
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+            const uint32_t wcode = ((c < 4 ? r.w.x : r.w.y) >> ((c & 3) * 8)) & 0xFFu;
+            const uint32_t ucode = (uw[c >> 1] >> ((c & 1) * 16)) & 0xFFFFu;
+            y[c] = sum16(wcode, ucode);
+        }
+    }
+    __device__ __forceinline__ uint32_t exact_bits(const Regs&, int, float y) const { return arith_bits(y); }
+    __device__ __forceinline__ uint32_t scalar(size_t i) const
+    {
+        return arith_bits(sum16(static_cast<const uint8_t*>(w8)[i], static_cast<const uint16_t*>(u16)[i]));
+    }
+};
+
 // ---------------------------------------------------------------------------- packing a row of codes
 // Fast rows: t[] as left by round_row_fast (bfloat16: code in bits 16..31 with the sign;
 // other formats: magnitude code, sign still to be taken from y).
@@ -351,6 +395,7 @@ tile_kernel(const Op op, void* __restrict__ dst, const uint64_t n_tiles, const u
             const uint32_t k0, const uint32_t k1, const uint32_t* __restrict__ words, const uint32_t tail_count)
 {
     using T = Tile<K>;
+    constexpr bool DRAWS = VAR < RTNE;                     // the deterministic modes use no random bits
     // The elements after the last whole tile (fewer than one tile) are done by CTA 0, one element per
     // thread and step, each with its own generator call: it starts first and overlaps the tiles.
     const uint32_t first_tile_cta = tail_count ? 1u : 0u;
@@ -359,8 +404,9 @@ tile_kernel(const Op op, void* __restrict__ dst, const uint64_t n_tiles, const u
         for (uint32_t i = threadIdx.x; i < tail_count; i += CTA_THREADS) {
             const size_t p = tail_begin + i;
             const uint32_t j = (uint32_t)(p % T::E);
-            uint32_t word;
-            if constexpr (BITS) {
+            uint32_t word = 0u;
+            if constexpr (!DRAWS) {
+            } else if constexpr (BITS) {
                 word = words[p / T::DPW];
             } else {
                 const uint4 o = philox_block(call0 + p / T::E, k0, k1);
@@ -382,7 +428,8 @@ tile_kernel(const Op op, void* __restrict__ dst, const uint64_t n_tiles, const u
         const size_t e0 = (size_t)tile * T::ELEMS;
         const uint64_t tile_call0 = call0 + tile * T::CALLS;
 
-        if constexpr (BITS) {
+        if constexpr (!DRAWS) {
+        } else if constexpr (BITS) {
             const uint32_t* src_words = words + tile * T::WORDS;
 #pragma unroll
             for (int j = 0; j < T::WORDS / 32; ++j) wb[j * 32 + lane] = __ldg(src_words + j * 32 + lane);
@@ -414,8 +461,12 @@ tile_kernel(const Op op, void* __restrict__ dst, const uint64_t n_tiles, const u
                     float y[8];
                     op.finish(e0 + p0, regs[j], y);
                     Draws8<K> d;
-                    if constexpr (OWN_CALL) d.from_call(philox_block(tile_call0 + (rb + j) * 32 + lane, k0, k1));
-                    else d.from_stream(wb, p0);
+                    if constexpr (!DRAWS) {
+                    } else if constexpr (OWN_CALL) {
+                        d.from_call(philox_block(tile_call0 + (rb + j) * 32 + lane, k0, k1));
+                    } else {
+                        d.from_stream(wb, p0);
+                    }
                     uint32_t t[8];
                     const bool redo = round_row_fast<FMT, VAR, K>(y, d, t);
                     if (!redo) {
@@ -432,7 +483,7 @@ tile_kernel(const Op op, void* __restrict__ dst, const uint64_t n_tiles, const u
                 }
             }
         }
-        if constexpr (!OWN_CALL) __syncwarp();      // the buffer is rewritten by the next tile
+        if constexpr (DRAWS && !OWN_CALL) __syncwarp();      // the buffer is rewritten by the next tile
     }
 }
 

@@ -52,7 +52,7 @@ def test_argument_validation_needs_no_device(lib):
     lib.fbsr_round.argtypes = [vp, vp, sz, i, i, i, u64, u64, f, vp]
     # invalid enum / k / scale are rejected before anything touches the device
     assert lib.fbsr_round(None, None, 0, 9, 0, 4, 0, 0, 1.0, None) == 1
-    assert lib.fbsr_round(None, None, 0, 0, 3, 4, 0, 0, 1.0, None) == 1
+    assert lib.fbsr_round(None, None, 0, 0, 6, 4, 0, 0, 1.0, None) == 1
     assert lib.fbsr_round(None, None, 0, 0, 0, 0, 0, 0, 1.0, None) == 1
     assert lib.fbsr_round(None, None, 0, 0, 0, 17, 0, 0, 1.0, None) == 1
     assert lib.fbsr_round(None, None, 0, 0, 0, 4, 0, 0, -1.0, None) == 1
