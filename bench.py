@@ -300,6 +300,32 @@ def main():
                 t8["%s/srf/k%d" % (fmt, k)] = round(5.0 * (1 << 27) / (a.elapsed_time(b) / 10 * 1e-3) / 1e9, 1)
         extras["round_fp8_GBps"] = t8
         del x8, out8
+        # 16-bit sources into 8-bit formats (3 B/element) and the 16-bit-sum weight update (4 B/element)
+        codes16 = workloads.lp_sweep(n_local, "bf16", device=dev)
+        w8 = torch.empty(n_local, dtype=torch.uint8, device=dev)
+        tlp = {}
+        for fmt in ("e4m3", "e5m2"):
+            for variant in VARIANT_LIST:
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                fbsr.fbsr_round_lp(codes16, "bf16", fmt, variant, 3, seed=SEED, out=w8)
+                a.record(stream)
+                for _ in range(10):
+                    fbsr.fbsr_round_lp(codes16, "bf16", fmt, variant, 3, seed=SEED, out=w8)
+                b.record(stream)
+                torch.cuda.synchronize()
+                tlp["bf16->%s/%s/k3" % (fmt, variant)] = round(3.0 * n_local / (a.elapsed_time(b) / 10 * 1e-3) / 1e9, 1)
+        extras["round_lp_GBps"] = tlp
+        fbsr.fbsr_round_lp(codes16, "bf16", "e4m3", "rtne", 1, seed=0, out=w8)
+        upd = (torch.randn(n_local, device=dev) * 0.01).to(torch.bfloat16).view(torch.uint16)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        fbsr.fbsr_qat_update(w8, upd, "e4m3", "bf16", "src", 3, seed=1)
+        a.record(stream)
+        for s_ in range(10):
+            fbsr.fbsr_qat_update(w8, upd, "e4m3", "bf16", "src", 3, seed=2 + s_)
+        b.record(stream)
+        torch.cuda.synchronize()
+        extras["qat_update_e4m3_bf16_src_k3_GBps"] = round(4.0 * n_local / (a.elapsed_time(b) / 10 * 1e-3) / 1e9, 1)
+        del codes16, w8, upd
         # fused optimizer step on the 32-block parameter list (22 B/param SGD-momentum, 30 B/param Adam)
         try:
             n_p = workloads.optimizer_param_count(32)

@@ -156,6 +156,27 @@ int by_variant_and_k(const Op& op, const CallArgs& a)
 #define FBSR_CAT(a, b) FBSR_CAT_(a, b)
 
 #if FBSR_GROUP == 0
+namespace {
+template <int K>
+void launch_stats_rows(const CallArgs& a, uint64_t n_rows, int n_ctas)
+{
+    stats_row_kernel<FMT, K><<<(unsigned)n_ctas, CTA_THREADS, 0, a.stream>>>(
+        a.src, a.scale, a.dst, n_rows, a.offset, a.variant, (uint32_t)a.seed, (uint32_t)(a.seed >> 32), a.group_size,
+        a.gsum_e, a.gsum_e2, static_cast<StatsAcc*>(a.partials));
+}
+template <int... Ks>
+void stats_rows_dispatch(const CallArgs& a, uint64_t n_rows, int n_ctas, std::integer_sequence<int, Ks...>)
+{
+    using Fn = void (*)(const CallArgs&, uint64_t, int);
+    static constexpr Fn table[16] = {&launch_stats_rows<Ks + 1>...};
+    table[a.k - 1](a, n_rows, n_ctas);
+}
+inline void stats_rows_by_k(const CallArgs& a, uint64_t n_rows, int n_ctas)
+{
+    stats_rows_dispatch(a, n_rows, n_ctas, std::make_integer_sequence<int, 16>{});
+}
+}  // namespace
+
 int FBSR_CAT(dispatch_round_, FBSR_FMT)(const CallArgs& a)
 {
     const RoundOp op{a.src, a.scale};
@@ -163,9 +184,23 @@ int FBSR_CAT(dispatch_round_, FBSR_FMT)(const CallArgs& a)
     case OP_ROUND: return by_variant_and_k<RoundOp, false>(op, a);
     case OP_ROUND_BITS: return by_variant_and_k<RoundOp, true>(op, a);
     case OP_ROUND_STATS: {
-        // Statistics run on the general kernel only; per-CTA partials are reduced in a fixed order.
+        // Whole rows of 256 elements go to the row kernel when the pointers allow vector access, the rest to
+        // the general kernel; each CTA leaves one partial in the workspace and they are summed in a fixed order.
         int n_ctas = 0;
-        launch_generic<RoundOp, false, true>(op, a, 0, a.n, &n_ctas);
+        uint64_t n_rows = 0;
+        if (aligned(a.src, 32) && aligned(a.dst, CODE_BYTES == 2 ? 16 : 8)) n_rows = a.n / ROW_ELEMS;
+        if (n_rows > 0) {
+            const uint64_t want = (n_rows + WARPS_PER_CTA - 1) / WARPS_PER_CTA;
+            const uint64_t cap = MAX_SLOW_GRID - 8;                 // the last slots belong to the ragged end
+            n_ctas = (int)(want < cap ? want : cap);
+            stats_rows_by_k(a, n_rows, n_ctas);
+            count_launch();
+        }
+        CallArgs rest = a;
+        rest.partials = static_cast<StatsAcc*>(a.partials) + n_ctas;
+        int rest_ctas = 0;
+        launch_generic<RoundOp, false, true>(op, rest, n_rows * ROW_ELEMS, a.n, &rest_ctas);
+        n_ctas += rest_ctas;
         stats_finalize_kernel<<<1, CTA_THREADS, 0, a.stream>>>(static_cast<const StatsAcc*>(a.partials), n_ctas,
                                                                static_cast<StatsAcc*>(a.total));
         count_launch();

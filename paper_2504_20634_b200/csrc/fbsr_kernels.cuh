@@ -606,6 +606,78 @@ generic_kernel(const Op op, void* __restrict__ dst, const uint64_t i_begin, cons
     }
 }
 
+// Statistics on aligned rows: a warp takes rows of 256 elements (one 256-bit load and one packed store per
+// lane), every lane computes the one or two generator calls that cover its 8 elements, rounds them with the
+// element-wise integer rounder and accumulates e = up - delta in binary64.  Any `offset` is served, because
+// the draws are located from the global index; only the pointers must be vector-aligned.
+template <int FMT, int K>
+__global__ void __launch_bounds__(CTA_THREADS)
+stats_row_kernel(const float* __restrict__ src, const float scale, void* __restrict__ dst, const uint64_t n_rows,
+                 const uint64_t offset, const int variant, const uint32_t k0, const uint32_t k1,
+                 const uint64_t group_size, double* __restrict__ gsum_e, double* __restrict__ gsum_e2,
+                 StatsAcc* __restrict__ partials)
+{
+    using T = Tile<K>;
+    static_assert(T::E >= 8, "a lane's 8 elements span at most two generator calls");
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const bool draws = variant < RTNE;
+    StatsAcc acc;
+    stats_zero(acc);
+    for (uint64_t row = (uint64_t)blockIdx.x * WARPS_PER_CTA + warp; row < n_rows;
+         row += (uint64_t)gridDim.x * WARPS_PER_CTA) {
+        const uint64_t i0 = row * ROW_ELEMS + lane * 8;
+        float x[8];
+        unpack(load_f8_stream(src + i0), x);
+        const uint64_t g0 = offset + i0, call = g0 / T::E;
+        const uint32_t j0 = (uint32_t)(g0 - call * T::E);
+        uint4 a = make_uint4(0u, 0u, 0u, 0u), b = a;
+        if (draws) {
+            a = philox_block(call, k0, k1);
+            b = (j0 + 7 >= (uint32_t)T::E) ? philox_block(call + 1, k0, k1) : a;
+        }
+        uint64_t grp = 0, grp_end = ~0ull;
+        double ge = 0.0, ge2 = 0.0;
+        if (group_size) { grp = i0 / group_size; grp_end = (grp + 1) * group_size; }
+        uint32_t codes[8];
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+            uint32_t j = j0 + c;
+            const uint4 o = j < (uint32_t)T::E ? a : b;
+            j = j < (uint32_t)T::E ? j : j - T::E;
+            const uint32_t ws = j / T::DPW;
+            const uint32_t word = ws == 0 ? o.x : ws == 1 ? o.y : ws == 2 ? o.z : o.w;
+            const uint32_t n = (word >> ((j % T::DPW) * K)) & T::MASK;
+            const uint32_t y = scaled_bits(x[c], scale);
+            ElementInfo info;
+            codes[c] = round_core<FMT, true>(y, n, variant, K, &info);
+            if (info.kind == 0) {
+                const double e = (double)info.up - info.delta, e2 = e * e;
+                acc.n_finite += 1; acc.n_up += (unsigned)info.up;
+                acc.sum_e += e; acc.sum_e2 += e2;
+                acc.sum_signed_e += (y >> 31) ? -e : e;
+                acc.sum_abs_e += fabs(e);
+                if (group_size) {
+                    while (i0 + c >= grp_end) {               // this element starts a later group: flush
+                        if (ge != 0.0 || ge2 != 0.0) { atomicAdd(gsum_e + grp, ge); atomicAdd(gsum_e2 + grp, ge2); }
+                        ge = 0.0; ge2 = 0.0;
+                        grp = (i0 + c) / group_size; grp_end = (grp + 1) * group_size;
+                    }
+                    ge += e; ge2 += e2;
+                }
+            } else if (info.kind == 1) acc.n_nan += 1;
+            else if (info.kind == 2) acc.n_inf += 1;
+            else acc.n_sat += 1;
+        }
+        if (group_size && (ge != 0.0 || ge2 != 0.0)) {
+            // the group of the row's last SR-rounded element
+            atomicAdd(gsum_e + grp, ge); atomicAdd(gsum_e2 + grp, ge2);
+        }
+        store_codes8<FMT>(dst, i0, codes);
+    }
+    stats_cta_reduce(acc);
+    if (threadIdx.x == 0) partials[blockIdx.x] = acc;
+}
+
 // Sum the per-CTA partials in a fixed order into the caller's fbsr_stats (same layout as StatsAcc).
 static __global__ void __launch_bounds__(CTA_THREADS)
 stats_finalize_kernel(const StatsAcc* __restrict__ partials, const int n_partials, StatsAcc* __restrict__ total)
