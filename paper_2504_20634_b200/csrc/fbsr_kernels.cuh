@@ -269,6 +269,26 @@ struct AdamOp {
     }
 };
 
+// Four stored 8-bit codes (one 32-bit word, low byte first) widened exactly to binary32 (Eq. (1)) by way of
+// binary16, which holds every value of both 8-bit formats: E5M2 is the upper byte of a binary16 pattern,
+// E4M3 has a hardware convert for pairs.  NaN codes become NaNs (the sign rule is applied by the caller).
+template <int FMT>
+__device__ __forceinline__ void decode4(uint32_t w, float (&v)[4])
+{
+    static_assert(FMT == E4M3 || FMT == E5M2, "8-bit formats");
+    uint32_t h01, h23;
+    if constexpr (FMT == E5M2) {
+        h01 = __byte_perm(w, 0u, 0x1404);                  // bytes [0, b0, 0, b1]
+        h23 = __byte_perm(w, 0u, 0x3424);                  // bytes [0, b2, 0, b3]
+    } else {
+        asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h01) : "h"((unsigned short)(w & 0xFFFFu)));
+        asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h23) : "h"((unsigned short)(w >> 16)));
+    }
+    const float2 a = __half22float2(*reinterpret_cast<const __half2*>(&h01));
+    const float2 b = __half22float2(*reinterpret_cast<const __half2*>(&h23));
+    v[0] = a.x; v[1] = a.y; v[2] = b.x; v[3] = b.y;
+}
+
 // y = fl32(value(w_lp) + u); the codes are rewritten in place by the caller of finish()
 template <int FMT>
 struct AccumOp {
@@ -291,12 +311,18 @@ struct AccumOp {
         float uv[8];
         unpack(r.u, uv);
         const uint32_t cw[4] = {r.c.x, r.c.y, r.c.z, r.c.w};
+        if constexpr (Format<FMT>::K == 8) {
+            float lo[4], hi[4];
+            decode4<FMT>(cw[0], lo);
+            decode4<FMT>(cw[1], hi);
 #pragma unroll
-        for (int c = 0; c < 8; ++c) {
-            uint32_t code;
-            if constexpr (Format<FMT>::K == 16) code = (cw[c >> 1] >> ((c & 1) * 16)) & 0xFFFFu;
-            else code = (cw[c >> 2] >> ((c & 3) * 8)) & 0xFFu;
-            y[c] = __fadd_rn(decode_element<FMT>(code), uv[c]);
+            for (int c = 0; c < 4; ++c) { y[c] = __fadd_rn(lo[c], uv[c]); y[c + 4] = __fadd_rn(hi[c], uv[c + 4]); }
+        } else {
+#pragma unroll
+            for (int c = 0; c < 8; ++c) {
+                const uint32_t code = (cw[c >> 1] >> ((c & 1) * 16)) & 0xFFFFu;
+                y[c] = __fadd_rn(decode_element<FMT>(code), uv[c]);
+            }
         }
     }
     __device__ __forceinline__ uint32_t scalar(size_t i) const
@@ -317,7 +343,10 @@ struct QatOp {
     struct Regs { uint2 w; uint4 u; };
     __device__ __forceinline__ static float sum16(uint32_t wcode, uint32_t ucode)
     {
-        const float wv = decode_element<WF>(wcode);
+        return sum16v(decode_element<WF>(wcode), ucode);
+    }
+    __device__ __forceinline__ static float sum16v(float wv, uint32_t ucode)
+    {
         const float uv = UF == BF16 ? __uint_as_float(ucode << 16) : __half2float(__ushort_as_half((unsigned short)ucode));
         float s = __fadd_rn(wv, uv);
         // round to the 16-bit format, ties to even; a finite sum beyond its largest value saturates
@@ -337,11 +366,13 @@ struct QatOp {
     __device__ __forceinline__ void finish(size_t, const Regs& r, float (&y)[8]) const
     {
         const uint32_t uw[4] = {r.u.x, r.u.y, r.u.z, r.u.w};
+        float lo[4], hi[4];
+        decode4<WF>(r.w.x, lo);
+        decode4<WF>(r.w.y, hi);
 #pragma unroll
         for (int c = 0; c < 8; ++c) {
-            const uint32_t wcode = ((c < 4 ? r.w.x : r.w.y) >> ((c & 3) * 8)) & 0xFFu;
             const uint32_t ucode = (uw[c >> 1] >> ((c & 1) * 16)) & 0xFFFFu;
-            y[c] = sum16(wcode, ucode);
+            y[c] = sum16v(c < 4 ? lo[c] : hi[c - 4], ucode);
         }
     }
     __device__ __forceinline__ uint32_t exact_bits(const Regs&, int, float y) const { return arith_bits(y); }
