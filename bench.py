@@ -359,6 +359,14 @@ def main():
         cpu_baseline = {"value": sample * len(combos) / sec / 1e9, "unit": UNIT, "cores": threads, "kind": "oracle",
                         "sample": "first 2^22 elements of the sweep tensor, all 48 (format, variant, k) combinations, once",
                         "host_cores_available": os.cpu_count()}
+        # the same oracle on every host core (disjoint chunks, global index as offset), a larger sample
+        all_threads = max(1, os.cpu_count() or 1)
+        if all_threads > 1:
+            big = min(n_local, (1 << 22) * min(all_threads, 8))
+            xb = x[:big].cpu().numpy()
+            sec_all = time_oracle(xb, combos, offset, all_threads)
+            cpu_baseline["all_cores"] = {"value": big * len(combos) / sec_all / 1e9, "unit": UNIT, "cores": all_threads,
+                                         "sample": "first %d elements, all 48 combinations, once" % big}
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                 "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
                 "vs_baseline": None, "dtype": "u32", "data": "synthetic",

@@ -161,7 +161,10 @@ __device__ __forceinline__ uint32_t round_core(uint32_t ybits, uint32_t n, const
 template <int K> struct Draws8 {
     static constexpr int DPW = 32 / K;
     static constexpr bool POW2 = (DPW & (DPW - 1)) == 0;
-    static constexpr int G = POW2 ? (DPW >= 8 ? 8 : DPW) : (4 * K <= 32 ? 4 : 2);
+    // fields per normalised word: a whole group must fit in 32 bits and, when two neighbouring words are
+    // joined, inside those two words for every starting field (f + G <= 2 dpw)
+    static constexpr int G = POW2 ? (DPW >= 8 ? 8 : DPW)
+                                  : (8 * K <= 32 && DPW >= 7) ? 8 : (4 * K <= 32 ? 4 : 2);
     static constexpr uint32_t MASK = (1u << K) - 1u;
     uint32_t u[8 / G] = {};
 
