@@ -129,7 +129,7 @@ static uint32_t field_of_words(const uint32_t* words, size_t i, int k)
 /* ------------------------------------------------------------- Eq. (1) */
 float fbsr_oracle_decode(int fmt, uint32_t code)
 {
-    const format_t* f = &FORMATS[fmt];
+    const format_t* f = &FORMATS[fmt & 0xFF];
     uint32_t s = (code >> (f->K - 1)) & 1u;
     uint32_t e = (code >> (f->P - 1)) & ((1u << (f->K - f->P)) - 1u);
     uint32_t t = code & ((1u << (f->P - 1)) - 1u);
@@ -147,6 +147,11 @@ float fbsr_oracle_decode(int fmt, uint32_t code)
 uint32_t fbsr_oracle_round_one(float y, int fmt, int variant, int N, uint32_t n,
                                int* kind_out, int* up_out, double* delta_out)
 {
+    /* bit 8 of fmt selects the paper-literal treatment of finite values beyond M (Section II: "rounded
+       deterministically as in IEEE-754 round to nearest"): below M + ulp(M)/2 they give M, from there on
+       the infinity (the NaN code where the format has no infinity).  Without it they saturate to M. */
+    const int ieee_overflow = (fmt >> 8) & 1;
+    fmt &= 0xFF;
     const format_t* f = &FORMATS[fmt];
     const int P = f->P, B = f->B;
     uint32_t yb = bits_of(y);
@@ -159,7 +164,18 @@ uint32_t fbsr_oracle_round_one(float y, int fmt, int variant, int N, uint32_t n,
     if (mag > 0x7F800000u) { kind = KIND_NAN; code = f->nan_code; goto done; }
     if (mag == 0x7F800000u) { kind = KIND_INF; code = f->has_inf ? f->inf_code : f->max_code; goto done; }
     if (mag == 0u) { code = 0u; goto done; }
-    if ((double)fabsf(y) > f->M) { kind = KIND_SAT; code = f->max_code; goto done; }
+    if ((double)fabsf(y) > f->M) {
+        kind = KIND_SAT; code = f->max_code;
+        if (ieee_overflow) {
+            int e2;
+            frexp(f->M, &e2);                                    /* M = m 2^e2, m in [0.5, 1) */
+            const double half_ulp = ldexp(1.0, (e2 - 1) - (f->P - 1) - 1);
+            /* exactly M + ulp/2 is a tie: it goes to the even neighbour, which is M when M's last bit is 0 */
+            const double a = (double)fabsf(y), thr = f->M + half_ulp;
+            if (a > thr || (a == thr && (f->max_code & 1u))) code = f->has_inf ? f->inf_code : f->nan_code;
+        }
+        goto done;
+    }
 
     {
         /* |y| = m * 2^q exactly, m the 24-bit integer significand. */
@@ -222,13 +238,13 @@ done:
 
 static void store_code(void* dst, size_t i, int fmt, uint32_t code)
 {
-    if (FORMATS[fmt].K == 16) ((uint16_t*)dst)[i] = (uint16_t)code;
+    if (FORMATS[fmt & 0xFF].K == 16) ((uint16_t*)dst)[i] = (uint16_t)code;
     else ((uint8_t*)dst)[i] = (uint8_t)code;
 }
 
 static uint32_t load_code(const void* src, size_t i, int fmt)
 {
-    return FORMATS[fmt].K == 16 ? ((const uint16_t*)src)[i] : ((const uint8_t*)src)[i];
+    return FORMATS[fmt & 0xFF].K == 16 ? ((const uint16_t*)src)[i] : ((const uint8_t*)src)[i];
 }
 
 /* y = fl32(x * scale), one rounded binary32 multiply (scaled tensors,
@@ -242,7 +258,7 @@ static float arith_result(float y) { return isnan(y) ? NAN : y; }
 
 static int bad_args(int fmt, int variant, int k)
 {
-    return fmt < 0 || fmt > 3 || variant < 0 || variant > 5 || k < 1 || k > 16;
+    return (fmt & ~0x100) < 0 || (fmt & ~0x100) > 3 || variant < 0 || variant > 5 || k < 1 || k > 16;
 }
 
 /* ------------------------------------------------------------ array forms */
@@ -387,7 +403,7 @@ int fbsr_oracle_adam_update(float* w, const float* g, float* m, float* v, void* 
 int fbsr_oracle_qat_update(void* w8, const void* u16, size_t n, int w_fmt, int u_fmt, int variant, int k,
                            uint64_t seed, uint64_t offset)
 {
-    if (bad_args(w_fmt, variant, k) || u_fmt < 0 || u_fmt > 1 || w_fmt < 2) return 1;
+    if (bad_args(w_fmt, variant, k) || u_fmt < 0 || u_fmt > 1 || (w_fmt & 0xFF) < 2) return 1;
     for (size_t i = 0; i < n; ++i) {
         float wv = fbsr_oracle_decode(w_fmt, load_code(w8, i, w_fmt));
         float uv = fbsr_oracle_decode(u_fmt, load_code(u16, i, u_fmt));

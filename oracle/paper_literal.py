@@ -230,7 +230,7 @@ def round_positive(xt, fmt, variant, n, N):
     return code, up, delta
 
 
-def round_f32_bits(ybits, fmt, variant, n, N):
+def round_f32_bits(ybits, fmt, variant, n, N, ieee_overflow=False):
     """Round one binary32 pattern (already scaled) to the target format.
 
     Policy outside the paper's scope (Section II says such values are handled
@@ -254,6 +254,13 @@ def round_f32_bits(ybits, fmt, variant, n, N):
         return sign, "finite", 0, Fraction(0)
     xt = f32_bits_to_fraction(mag)
     if xt > f["M"]:
+        if ieee_overflow:
+            # Section II: values beyond the finite range are rounded as IEEE round-to-nearest does:
+            # M below M + ulp(M)/2, the infinity (or the NaN of a format without one) above it, ties to even.
+            half_ulp = pow2(floor_log2(f["M"]) - (f["P"] - 1) - 1)
+            thr = f["M"] + half_ulp          # a tie at thr goes to the even neighbour: M if its last bit is 0
+            if xt > thr or (xt == thr and f["max_code"] & 1):
+                return sign | (f["inf_code"] if f["inf_code"] is not None else f["nan_code"]), "sat", 0, Fraction(0)
         return sign | f["max_code"], "sat", 0, Fraction(0)
     code, up, delta = round_positive(xt, fmt, variant, n, N)
     return sign | code, "finite", up, delta

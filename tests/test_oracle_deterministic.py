@@ -68,3 +68,33 @@ def test_qat_update_composition_and_stagnation():
     tiny = (wv * 0.01).astype(np.float32)                            # far below half an e4m3 ulp
     t16 = torch.from_numpy(tiny).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
     assert np.array_equal(capi.qat_update(w8.copy(), t16, "e4m3", "bf16", "rtne", 1, seed=0), w8)
+
+
+@pytest.mark.parametrize("fmt", FMTS)
+def test_paper_literal_overflow_option(fmt):
+    """With the IEEE-overflow flag, nearest-even rounding of finite values beyond M matches torch's cast
+    (M below M + ulp/2, then Inf; NaN for E4M3, which has no infinity); stochastic variants treat those
+    values the same way, and in-range values are unaffected by the flag."""
+    M = float(pl.FORMATS[fmt]["M"])
+    M32 = np.float32(M)
+    ulp = M32 - np.nextafter(M32, np.float32(0)) if fmt != "bf16" else np.float32(2.0 ** 120)
+    ulp = np.float32(2.0 ** (np.floor(np.log2(M)) - (pl.FORMATS[fmt]["P"] - 1)))
+    xs = np.array([M, np.nextafter(M32, np.float32(np.inf)), M + 0.49 * ulp, np.nextafter(np.float32(M + 0.5 * ulp), np.float32(0)),
+                   M + 0.5 * ulp, M + 0.75 * ulp, M * 1.5, -(M + 0.5 * ulp), -(M + 0.25 * ulp)], dtype=np.float32)
+    xs = xs[np.isfinite(xs)]
+    got = capi.fbsr_round(xs, fmt + "+ieee", "rtne", 1, seed=0)
+    t = torch.from_numpy(xs.copy()).to(TORCH_DTYPE[fmt])
+    expect = t.view(torch.int16 if got.dtype == np.uint16 else torch.uint8).numpy().view(got.dtype)
+    if fmt == "e4m3":
+        # torch's NaN code carries the sign; ours too
+        assert np.array_equal(got & 0x7F, expect & 0x7F)
+    else:
+        assert np.array_equal(got, expect)
+    for variant in ("srff", "srf", "src"):
+        assert np.array_equal(capi.fbsr_round(xs, fmt + "+ieee", variant, 4, seed=3), got)
+    for i, x in enumerate(xs):
+        c0 = pl.round_f32_bits(int(np.float32(x).view(np.uint32)), fmt, "rtne", 0, 1, ieee_overflow=True)[0]
+        assert c0 == int(got[i])
+    rng = np.random.default_rng(44)
+    inr = (bits_f32(random_f32(rng, 2000, -10, 6))).astype(np.float32)
+    assert np.array_equal(capi.fbsr_round(inr, fmt + "+ieee", "srf", 3, seed=1), capi.fbsr_round(inr, fmt, "srf", 3, seed=1))
