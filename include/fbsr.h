@@ -66,6 +66,12 @@ typedef enum {
     FBSR_E5M2 = 3  /* ( 8,  3,  15; 57344) */
 } fbsr_fmt;
 
+/* May be or-ed into any `fmt` argument.  Section II says that values beyond the finite range are "rounded
+ * deterministically as in IEEE-754 round to nearest"; with this flag finite |y| > M follow that reading
+ * (M below M + ulp(M)/2, +-Inf above it -- the NaN code for e4m3 -- ties to the even neighbour) instead
+ * of saturating.  Calls with the flag run on the general (slower) kernel. */
+#define FBSR_OVF_IEEE 0x100
+
 /* Round-up predicates: the few-bit stochastic ones of Section II-B and Eq. (8), and the deterministic
  * ones of Section II-A (ties to even, ties away from zero (Eq. (4)), ties to odd), which use no draw:
  * for those k_bits, seed and offset are ignored (k_bits must still be in 1..16). */

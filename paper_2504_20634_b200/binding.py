@@ -14,6 +14,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_HERE, "libfbsr.so")
 
 FMT = {"bf16": 0, "fp16": 1, "e4m3": 2, "e5m2": 3}
+OVF_IEEE = 0x100          # or into a format id, or append "+ieee" to a format name: IEEE overflow instead of saturation
 VARIANT = {"srff": 0, "srf": 1, "src": 2, "rtne": 3, "rta": 4, "rto": 5}
 CODE_DTYPE = {"bf16": torch.uint16, "fp16": torch.uint16, "e4m3": torch.uint8, "e5m2": torch.uint8}
 VIEW_DTYPE = {"bf16": torch.bfloat16, "fp16": torch.float16, "e4m3": torch.float8_e4m3fn,
@@ -101,12 +102,16 @@ def fbsr_round_host_min_workspace():
 
 
 def _fmt(fmt):
-    return fmt if isinstance(fmt, int) else FMT[fmt]
+    if isinstance(fmt, int):
+        return fmt
+    return FMT[fmt[:-5]] | OVF_IEEE if fmt.endswith("+ieee") else FMT[fmt]
 
 
 def _fmt_name(fmt):
     # unknown integers fall through to the library, which rejects them with a status code
-    return fmt if isinstance(fmt, str) else {v: k for k, v in FMT.items()}.get(fmt, "bf16")
+    if isinstance(fmt, str):
+        return fmt[:-5] if fmt.endswith("+ieee") else fmt
+    return {v: k for k, v in FMT.items()}.get(fmt & ~OVF_IEEE, "bf16")
 
 
 def _var(variant):

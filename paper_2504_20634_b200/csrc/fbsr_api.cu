@@ -19,6 +19,13 @@ const dispatch_fn kRound[4] = {dispatch_round_0, dispatch_round_1, dispatch_roun
 const dispatch_fn kOptim[4] = {dispatch_optim_0, dispatch_optim_1, dispatch_optim_2, dispatch_optim_3};
 
 inline bool bad_enum(int fmt, int variant, int k) { return fmt < 0 || fmt > 3 || variant < 0 || variant > 5 || k < 1 || k > 16; }
+// FBSR_OVF_IEEE may be or-ed into a format argument: take it out and report it.
+inline int take_overflow_flag(int& fmt)
+{
+    const int flag = (fmt & FBSR_OVF_IEEE) ? 1 : 0;
+    fmt &= ~FBSR_OVF_IEEE;
+    return flag;
+}
 inline size_t code_bytes(int fmt) { return fmt <= 1 ? 2 : 1; }
 inline bool misaligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) != 0; }
 
@@ -55,9 +62,11 @@ extern "C" {
 int fbsr_round(const float* src, void* dst, size_t n, int fmt, int variant, int k_bits, uint64_t seed,
                uint64_t offset, float scale, void* cuda_stream)
 {
+    const int ovf_ieee = take_overflow_flag(fmt);
     if (int rc = check_round(src, dst, n, fmt, variant, k_bits, scale)) return rc;
     if (n == 0) return FBSR_OK;
     CallArgs a = base_args(OP_ROUND, variant, k_bits, n, seed, offset, dst, cuda_stream);
+    a.ovf_ieee = ovf_ieee;
     a.src = src; a.scale = scale;
     return finish(kRound[fmt](a));
 }
@@ -65,6 +74,7 @@ int fbsr_round(const float* src, void* dst, size_t n, int fmt, int variant, int 
 int fbsr_round_lp(const void* src, int src_fmt, void* dst, size_t n, int dst_fmt, int variant, int k_bits,
                   uint64_t seed, uint64_t offset, float scale, void* cuda_stream)
 {
+    const int ovf_ieee = take_overflow_flag(dst_fmt);
     if (bad_enum(dst_fmt, variant, k_bits) || src_fmt < 0 || src_fmt > 3) return FBSR_ERR_INVALID_ARG;
     if (!(scale > 0.0f) || !std::isfinite(scale)) return FBSR_ERR_INVALID_ARG;
     if ((src_fmt != FBSR_BF16 && src_fmt != FBSR_FP16) || (dst_fmt != FBSR_E4M3 && dst_fmt != FBSR_E5M2))
@@ -73,6 +83,7 @@ int fbsr_round_lp(const void* src, int src_fmt, void* dst, size_t n, int dst_fmt
     if (misaligned(src, 2)) return FBSR_ERR_ALIGNMENT;
     if (n == 0) return FBSR_OK;
     CallArgs a = base_args(OP_ROUND_LP, variant, k_bits, n, seed, offset, dst, cuda_stream);
+    a.ovf_ieee = ovf_ieee;
     a.src_lp = src; a.src_fmt = src_fmt; a.scale = scale;
     return finish(dst_fmt == FBSR_E4M3 ? dispatch_lp_2(a) : dispatch_lp_3(a));
 }
@@ -80,11 +91,13 @@ int fbsr_round_lp(const void* src, int src_fmt, void* dst, size_t n, int dst_fmt
 int fbsr_round_bits(const float* src, void* dst, size_t n, int fmt, int variant, int k_bits,
                     const uint32_t* rand_words, float scale, void* cuda_stream)
 {
+    const int ovf_ieee = take_overflow_flag(fmt);
     if (int rc = check_round(src, dst, n, fmt, variant, k_bits, scale)) return rc;
     if (n > 0 && rand_words == nullptr) return FBSR_ERR_INVALID_ARG;
     if (misaligned(rand_words, 4)) return FBSR_ERR_ALIGNMENT;
     if (n == 0) return FBSR_OK;
     CallArgs a = base_args(OP_ROUND_BITS, variant, k_bits, n, 0, 0, dst, cuda_stream);
+    a.ovf_ieee = ovf_ieee;
     a.src = src; a.scale = scale; a.words = rand_words;
     return finish(kRound[fmt](a));
 }
@@ -95,6 +108,7 @@ int fbsr_round_stats(const float* src, void* dst, size_t n, int fmt, int variant
                      uint64_t offset, float scale, size_t group_size, double* group_sum_e, double* group_sum_e2,
                      fbsr_stats* total, void* workspace, size_t workspace_bytes, void* cuda_stream)
 {
+    const int ovf_ieee = take_overflow_flag(fmt);
     if (int rc = check_round(src, dst, n, fmt, variant, k_bits, scale)) return rc;
     if (total == nullptr) return FBSR_ERR_INVALID_ARG;
     if (group_size > 0 && n > 0 && (group_sum_e == nullptr || group_sum_e2 == nullptr)) return FBSR_ERR_INVALID_ARG;
@@ -102,6 +116,7 @@ int fbsr_round_stats(const float* src, void* dst, size_t n, int fmt, int variant
     if (workspace == nullptr || workspace_bytes < fbsr_stats_workspace_bytes()) return FBSR_ERR_WORKSPACE;
     if (misaligned(workspace, 8)) return FBSR_ERR_ALIGNMENT;
     CallArgs a = base_args(OP_ROUND_STATS, variant, k_bits, n, seed, offset, dst, cuda_stream);
+    a.ovf_ieee = ovf_ieee;
     a.src = src; a.scale = scale; a.group_size = group_size;
     a.gsum_e = group_sum_e; a.gsum_e2 = group_sum_e2; a.total = total; a.partials = workspace;
     if (group_size > 0 && n > 0) {
@@ -158,12 +173,14 @@ int fbsr_round_stats_noalloc(const float* src, void* dst, size_t n, int fmt, int
 int fbsr_sgd_update(float* master_w, const float* grad, float* momentum, void* dst_lp, size_t n, int fmt,
                     int variant, int k_bits, uint64_t seed, uint64_t offset, float lr, float mu, void* cuda_stream)
 {
+    const int ovf_ieee = take_overflow_flag(fmt);
     if (bad_enum(fmt, variant, k_bits)) return FBSR_ERR_INVALID_ARG;
     if (n > 0 && (!master_w || !grad || !momentum || !dst_lp)) return FBSR_ERR_INVALID_ARG;
     if (misaligned(master_w, 4) || misaligned(grad, 4) || misaligned(momentum, 4) ||
         misaligned(dst_lp, code_bytes(fmt))) return FBSR_ERR_ALIGNMENT;
     if (n == 0) return FBSR_OK;
     CallArgs a = base_args(OP_SGD, variant, k_bits, n, seed, offset, dst_lp, cuda_stream);
+    a.ovf_ieee = ovf_ieee;
     a.w = master_w; a.g = grad; a.m = momentum; a.neg_lr = -lr; a.mu = mu;
     return finish(kOptim[fmt](a));
 }
@@ -172,6 +189,7 @@ int fbsr_adam_update(float* master_w, const float* grad, float* m, float* v, voi
                      int variant, int k_bits, uint64_t seed, uint64_t offset, float lr, float beta1, float beta2,
                      float eps, int step, void* cuda_stream)
 {
+    const int ovf_ieee = take_overflow_flag(fmt);
     if (bad_enum(fmt, variant, k_bits) || step < 1) return FBSR_ERR_INVALID_ARG;
     if (n > 0 && (!master_w || !grad || !m || !v || !dst_lp)) return FBSR_ERR_INVALID_ARG;
     if (misaligned(master_w, 4) || misaligned(grad, 4) || misaligned(m, 4) || misaligned(v, 4) ||
@@ -181,6 +199,7 @@ int fbsr_adam_update(float* master_w, const float* grad, float* m, float* v, voi
     double b1t = 1.0, b2t = 1.0;
     for (int t = 0; t < step; ++t) { b1t *= (double)beta1; b2t *= (double)beta2; }
     CallArgs a = base_args(OP_ADAM, variant, k_bits, n, seed, offset, dst_lp, cuda_stream);
+    a.ovf_ieee = ovf_ieee;
     a.w = master_w; a.g = grad; a.m = m; a.v = v;
     a.beta1 = beta1; a.beta2 = beta2; a.eps = eps;
     a.neg_c1 = -(float)((double)lr / (1.0 - b1t));
@@ -193,11 +212,13 @@ int fbsr_adam_update(float* master_w, const float* grad, float* m, float* v, voi
 int fbsr_accumulate(void* w_lp, const float* update, size_t n, int fmt, int variant, int k_bits, uint64_t seed,
                     uint64_t offset, void* cuda_stream)
 {
+    const int ovf_ieee = take_overflow_flag(fmt);
     if (bad_enum(fmt, variant, k_bits)) return FBSR_ERR_INVALID_ARG;
     if (n > 0 && (!w_lp || !update)) return FBSR_ERR_INVALID_ARG;
     if (misaligned(update, 4) || misaligned(w_lp, code_bytes(fmt))) return FBSR_ERR_ALIGNMENT;
     if (n == 0) return FBSR_OK;
     CallArgs a = base_args(OP_ACCUM, variant, k_bits, n, seed, offset, w_lp, cuda_stream);
+    a.ovf_ieee = ovf_ieee;
     a.src = update;
     return finish(kOptim[fmt](a));
 }
@@ -205,12 +226,14 @@ int fbsr_accumulate(void* w_lp, const float* update, size_t n, int fmt, int vari
 int fbsr_qat_update(void* w8, const void* update16, size_t n, int w_fmt, int u_fmt, int variant, int k_bits,
                     uint64_t seed, uint64_t offset, void* cuda_stream)
 {
+    const int ovf_ieee = take_overflow_flag(w_fmt);
     if (bad_enum(w_fmt, variant, k_bits) || u_fmt < 0 || u_fmt > 3) return FBSR_ERR_INVALID_ARG;
     if ((w_fmt != FBSR_E4M3 && w_fmt != FBSR_E5M2) || (u_fmt != FBSR_BF16 && u_fmt != FBSR_FP16)) return FBSR_ERR_UNSUPPORTED;
     if (n > 0 && (!w8 || !update16)) return FBSR_ERR_INVALID_ARG;
     if (misaligned(update16, 2)) return FBSR_ERR_ALIGNMENT;
     if (n == 0) return FBSR_OK;
     CallArgs a = base_args(OP_QAT, variant, k_bits, n, seed, offset, w8, cuda_stream);
+    a.ovf_ieee = ovf_ieee;
     a.src_lp = update16; a.src_fmt = u_fmt;
     return finish(w_fmt == FBSR_E4M3 ? dispatch_lp_2(a) : dispatch_lp_3(a));
 }
@@ -231,6 +254,7 @@ int fbsr_round_host(const float* src_host, void* dst_host, size_t n, int fmt, in
                     uint64_t seed, uint64_t offset, float scale, void* dev_workspace, size_t workspace_bytes,
                     void* cuda_stream)
 {
+    const int ovf_ieee = take_overflow_flag(fmt);
     if (int rc = check_round(src_host, dst_host, n, fmt, variant, k_bits, scale)) return rc;
     if (dev_workspace == nullptr || workspace_bytes < fbsr_round_host_min_workspace()) return FBSR_ERR_WORKSPACE;
     if (misaligned(dev_workspace, 256)) return FBSR_ERR_ALIGNMENT;
@@ -282,6 +306,8 @@ int fbsr_round_host(const float* src_host, void* dst_host, size_t n, int fmt, in
         if (used[sl] && cudaStreamWaitEvent(main, s.drained[sl], 0) != cudaSuccess) return FBSR_ERR_CUDA;
         if (cudaMemcpyAsync(slot_in[sl], src_host + at, len * 4, cudaMemcpyHostToDevice, main) != cudaSuccess) return FBSR_ERR_CUDA;
         CallArgs a = base_args(OP_ROUND, variant, k_bits, len, seed, offset + at, slot_out[sl], main);
+        a.ovf_ieee = ovf_ieee;
+    a.ovf_ieee = ovf_ieee;
         a.src = reinterpret_cast<const float*>(slot_in[sl]); a.scale = scale;
         if (kRound[fmt](a) != 0) return FBSR_ERR_UNSUPPORTED;
         if (cudaEventRecord(s.rounded[sl], main) != cudaSuccess) return FBSR_ERR_CUDA;

@@ -86,7 +86,7 @@ struct ElementInfo {
 // ----------------------------------------------------------------------------
 template <int FMT, bool STATS>
 __device__ __forceinline__ uint32_t round_core(uint32_t ybits, uint32_t n, const int VAR, const int N,
-                                               ElementInfo* info)
+                                               ElementInfo* info, const bool ieee_overflow = false)
 {
     using F = Format<FMT>;
     constexpr int P = F::P;
@@ -148,7 +148,16 @@ __device__ __forceinline__ uint32_t round_core(uint32_t ybits, uint32_t n, const
     if (mag > F::MAXBITS) {
         if (mag > 0x7F800000u) { enc = F::NANCODE; if constexpr (STATS) info->kind = 1; }
         else if (mag == 0x7F800000u) { enc = F::INFCODE; if constexpr (STATS) info->kind = 2; }
-        else { enc = F::MAXCODE; if constexpr (STATS) info->kind = 3; }
+        else {
+            // finite and beyond M: saturate, or (Section II read literally) round as IEEE nearest-even does:
+            // M below M + ulp/2, the infinity above it (the NaN code for E4M3), the tie to the even neighbour
+            enc = F::MAXCODE;
+            if constexpr (STATS) info->kind = 3;
+            if (ieee_overflow) {
+                const uint32_t tie = F::MAXBITS + (1u << (24 - P - 1));
+                if (mag > tie || (mag == tie && (F::MAXCODE & 1u))) enc = FMT == E4M3 ? F::NANCODE : F::INFCODE;
+            }
+        }
     }
     return enc | sign;
 }

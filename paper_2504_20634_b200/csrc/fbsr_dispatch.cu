@@ -93,7 +93,7 @@ int launch_generic(const Op& op, const CallArgs& a, size_t i_begin, size_t i_end
     generic_kernel<Op, FMT, BITS, STATS><<<(unsigned)ctas, CTA_THREADS, 0, a.stream>>>(
         op, a.dst, i_begin, i_end, off, a.variant, a.k, (uint32_t)a.seed, (uint32_t)(a.seed >> 32),
         a.words, BITS ? (a.n + dpw - 1) / dpw : 0, STATS ? a.group_size : 0, a.gsum_e, a.gsum_e2,
-        static_cast<StatsAcc*>(a.partials));
+        static_cast<StatsAcc*>(a.partials), a.ovf_ieee);
     count_launch();
     if (n_ctas_out) *n_ctas_out = (int)ctas;
     return 0;
@@ -122,7 +122,8 @@ template <class Op, int VAR, int K, bool BITS>
 int run(const Op& op, const CallArgs& a)
 {
     const Plan p = make_plan<Op, K, BITS>(op, a);
-    if (p.n_tiles == 0) return launch_generic<Op, BITS, false>(op, a, 0, a.n, nullptr);
+    // the IEEE-overflow option is served by the general kernel only
+    if (p.n_tiles == 0 || a.ovf_ieee) return launch_generic<Op, BITS, false>(op, a, 0, a.n, nullptr);
     launch_generic<Op, BITS, false>(op, a, 0, p.head, nullptr);
     launch_tiles<Op, VAR, K, BITS>(op, a, p);          // whole tiles and the ragged end
     return 0;
@@ -188,7 +189,7 @@ int FBSR_CAT(dispatch_round_, FBSR_FMT)(const CallArgs& a)
         // the general kernel; each CTA leaves one partial in the workspace and they are summed in a fixed order.
         int n_ctas = 0;
         uint64_t n_rows = 0;
-        if (aligned(a.src, 32) && aligned(a.dst, CODE_BYTES == 2 ? 16 : 8)) n_rows = a.n / ROW_ELEMS;
+        if (!a.ovf_ieee && aligned(a.src, 32) && aligned(a.dst, CODE_BYTES == 2 ? 16 : 8)) n_rows = a.n / ROW_ELEMS;
         if (n_rows > 0) {
             const uint64_t want = (n_rows + WARPS_PER_CTA - 1) / WARPS_PER_CTA;
             const uint64_t cap = MAX_SLOW_GRID - 8;                 // the last slots belong to the ragged end

@@ -12,6 +12,7 @@ enum OpKind { OP_ROUND = 0, OP_ROUND_BITS, OP_ROUND_STATS, OP_SGD, OP_ADAM, OP_A
 struct CallArgs {
     OpKind op;
     int variant, k;
+    int ovf_ieee;                   // finite values beyond M: IEEE nearest-even instead of saturation
     size_t n;
     uint64_t seed, offset;
     cudaStream_t stream;

@@ -573,7 +573,7 @@ generic_kernel(const Op op, void* __restrict__ dst, const uint64_t i_begin, cons
                const uint64_t offset, const int variant, const int k, const uint32_t k0, const uint32_t k1,
                const uint32_t* __restrict__ words, const uint64_t n_words,
                const uint64_t group_size, double* __restrict__ gsum_e, double* __restrict__ gsum_e2,
-               StatsAcc* __restrict__ partials)
+               StatsAcc* __restrict__ partials, const int ieee_overflow)
 {
     const uint32_t dpw = 32u / (uint32_t)k, E = 4u * dpw, mask = (1u << k) - 1u;
     const uint64_t g_first = offset + i_begin, g_last = offset + i_end;     // [g_first, g_last)
@@ -604,7 +604,7 @@ generic_kernel(const Op op, void* __restrict__ dst, const uint64_t i_begin, cons
             const uint32_t n = (word >> (f * k)) & mask;
             const uint32_t y = op.scalar(i);
             ElementInfo info;
-            const uint32_t code = round_core<FMT, STATS>(y, n, variant, k, &info);
+            const uint32_t code = round_core<FMT, STATS>(y, n, variant, k, &info, ieee_overflow != 0);
             store_code1<FMT>(dst, i, code);
             if constexpr (STATS) {
                 if (info.kind == 0) {

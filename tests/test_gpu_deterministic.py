@@ -97,3 +97,30 @@ def test_section4_behaviour_in_miniature():
     assert abs(gain["src"] - exact) < tol
     assert abs(gain["srff"] - (exact - steps * 2.0 ** -5 * ulp)) < tol
     assert abs(gain["srf"] - (exact + steps * 2.0 ** -5 * ulp)) < tol
+
+
+@pytest.mark.parametrize("fmt", FMTS)
+def test_ieee_overflow_option(fmt):
+    """FBSR_OVF_IEEE: finite values beyond M follow IEEE nearest-even (M, then Inf / NaN) instead of saturating."""
+    rng = np.random.default_rng(97)
+    M = np.float32({"bf16": 3.3895313892515355e38, "fp16": 65504.0, "e4m3": 448.0, "e5m2": 57344.0}[fmt])
+    n = 6000
+    x = (M * (1.0 + rng.uniform(-0.2, 0.2, n))).astype(np.float32) * np.where(rng.integers(0, 2, n), 1, -1).astype(np.float32)
+    x[:100] = gu.mixed_inputs(100, 5, fmt)
+    P = {"bf16": 8, "fp16": 11, "e4m3": 4, "e5m2": 3}[fmt]
+    ulp = np.float32(2.0 ** (np.floor(np.log2(float(M))) - (P - 1)))
+    x[100:104] = [M + ulp / 2, -(M + ulp / 2), np.nextafter(np.float32(M + ulp / 2), np.float32(0)), np.nextafter(M, np.float32(np.inf))]
+    x = np.where(np.isinf(x), M, x).astype(np.float32)
+    xd = torch.from_numpy(x).cuda()
+    for variant, k in (("rtne", 1), ("srf", 3), ("src", 8)):
+        got = fbsr.fbsr_round(xd, fmt + "+ieee", variant, k, seed=2, offset=7)
+        gu.assert_codes_equal(got, capi.fbsr_round(x, fmt + "+ieee", variant, k, seed=2, offset=7), fmt + " ieee " + variant)
+        codes, st, _, _ = fbsr.fbsr_round_stats(xd, fmt + "+ieee", variant, k, seed=2, offset=7)
+        assert torch.equal(codes, got)
+    # nearest-even with the flag equals torch's cast on every finite input (torch overflows the same way)
+    got = fbsr.fbsr_round(xd, fmt + "+ieee", "rtne", 1, seed=0)
+    as_int = torch.int16 if got.dtype == torch.uint16 else torch.uint8
+    ref = xd.to(TORCH_DTYPE[fmt]).view(as_int)
+    mask = 0x7FFF if got.dtype == torch.uint16 else 0x7F
+    ok = torch.isfinite(xd)
+    assert torch.equal(got.view(as_int)[ok] & mask, ref[ok] & mask)
