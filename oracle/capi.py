@@ -69,6 +69,8 @@ def lib():
         vp, sz, i, u64, f = ctypes.c_void_p, ctypes.c_size_t, ctypes.c_int, ctypes.c_uint64, ctypes.c_float
         L.fbsr_oracle_round.argtypes = [vp, vp, sz, i, i, i, u64, u64, f]
         L.fbsr_oracle_round_bits.argtypes = [vp, vp, sz, i, i, i, vp, f]
+        L.fbsr_oracle_round_mx.argtypes = [vp, vp, vp, sz, i, i, i, u64, u64]
+        L.fbsr_oracle_round_mx.restype = ctypes.c_int
         L.fbsr_oracle_round_lp.argtypes = [vp, i, vp, sz, i, i, i, u64, u64, f]
         L.fbsr_oracle_round_lp.restype = ctypes.c_int
         L.fbsr_oracle_round_stats.argtypes = [vp, vp, sz, i, i, i, u64, u64, f, sz, vp, vp,
@@ -235,3 +237,13 @@ def qat_update(w8, u16, w_fmt, u_fmt, variant, k, seed, offset=0):
     _check(lib().fbsr_oracle_qat_update(_ptr(w8), _ptr(u16), w8.size, FMT[w_fmt], FMT[u_fmt], VARIANT[variant], k,
                                         seed, offset))
     return w8
+
+
+def fbsr_round_mx(src, fmt, variant, k, seed, offset=0):
+    """Block-scaled rounding (blocks of 32, shared power-of-two exponent); returns (codes, scale bytes)."""
+    src = _f32(src)
+    dst = np.empty(src.size, dtype=CODE_DTYPE[fmt])
+    scales = np.empty((src.size + 31) // 32, dtype=np.uint8)
+    _check(lib().fbsr_oracle_round_mx(_ptr(src), _ptr(dst), _ptr(scales), src.size, FMT[fmt], VARIANT[variant], k,
+                                      seed, offset))
+    return dst, scales

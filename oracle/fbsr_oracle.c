@@ -301,6 +301,43 @@ int fbsr_oracle_round_lp(const void* src, int src_fmt, void* dst, size_t n, int 
     return 0;
 }
 
+/* Block-scaled tensors (Section I-A: "blocks of low-precision values are accompanied by a scale factor,
+ * which may be a power of two").  Blocks are 32 consecutive elements of the call.  Per block:
+ *   amax = largest finite |x| (0 if none);  e_blk = clamp(floor(log2 amax) - emax, -127, 127) with
+ *   emax = floor(log2 M) of the target and e_blk = -127 for amax = 0 or subnormal;
+ *   scale byte = e_blk + 127;  y = fl32(x 2^-e_blk);  code = FBSR(y).
+ * The recipe (shared power-of-two exponent from the block maximum) is this library's definition. */
+int fbsr_oracle_round_mx(const float* src, void* dst, uint8_t* scales, size_t n, int fmt, int variant, int k,
+                         uint64_t seed, uint64_t offset)
+{
+    if (bad_args(fmt, variant, k)) return 1;
+    int emax;
+    frexp(FORMATS[fmt & 0xFF].M, &emax);
+    emax -= 1;                                            /* M = m 2^emax, m in [1, 2) */
+    for (size_t b0 = 0; b0 < n; b0 += 32) {
+        size_t b1 = b0 + 32 < n ? b0 + 32 : n;
+        float amax = 0.0f;
+        for (size_t i = b0; i < b1; ++i)
+            if (isfinite(src[i]) && fabsf(src[i]) > amax) amax = fabsf(src[i]);
+        int e_blk = -127;
+        if (amax >= 0x1p-126f) {
+            int e2;
+            frexpf(amax, &e2);                            /* amax = m 2^e2, m in [0.5, 1) */
+            e_blk = (e2 - 1) - emax;
+            if (e_blk < -127) e_blk = -127;
+            if (e_blk > 127) e_blk = 127;
+        }
+        scales[b0 / 32] = (uint8_t)(e_blk + 127);
+        const float s = ldexpf(1.0f, -e_blk);             /* exact, 2^-127 is a binary32 subnormal */
+        for (size_t i = b0; i < b1; ++i) {
+            float y = scaled(src[i], s);
+            uint32_t nr = fbsr_oracle_draw(seed, offset + i, k, 0u);
+            store_code(dst, i, fmt, fbsr_oracle_round_one(y, fmt, variant, k, nr, 0, 0, 0));
+        }
+    }
+    return 0;
+}
+
 /* Error of one SR-rounded element in target ulps: e = up - delta~ (the
  * quantity whose mean Section III calls bias).  Group g holds elements
  * [g*group_size, (g+1)*group_size) of this call. */
