@@ -118,6 +118,18 @@ int fbsr_round(const float* src, void* dst, size_t n, int fmt, int variant, int 
 int fbsr_round_lp(const void* src, int src_fmt, void* dst, size_t n, int dst_fmt, int variant, int k_bits,
                   uint64_t seed, uint64_t offset, float scale, void* cuda_stream);
 
+/* fbsr_round_mx -- block-scaled tensors (Section I-A: "blocks of low-precision values are accompanied by a
+ * scale factor, which may be a power of two").  Blocks are 32 consecutive elements of the call; per block
+ *     amax  = largest finite |src| (0 if none)
+ *     e_blk = clamp(floor(log2 amax) - emax, -127, 127), emax = floor(log2 M);  -127 if amax < 2^-126
+ *     scales[block] = e_blk + 127;   dst[i] = FBSR(fl32(src[i] * 2^-e_blk))
+ * so the block maximum lands in the format's top binade (values between M and 2^(emax+1) saturate).
+ *   scales   device, ceil(n / 32) bytes, overwritten
+ * Draws are indexed by offset + i as everywhere else.  The fast path additionally needs the first tile
+ * boundary of the call to fall on a block boundary (true for offset = 0 or any multiple of the tile size). */
+int fbsr_round_mx(const float* src, void* dst, uint8_t* scales, size_t n, int fmt, int variant, int k_bits,
+                  uint64_t seed, uint64_t offset, void* cuda_stream);
+
 /* fbsr_round_bits -- the same rounding with caller-supplied random bits
  * (Section II-B: "random numbers will be supplied as a finite sequence of random
  * bits").  rand_words: device, ceil(n / dpw) words; element i uses field

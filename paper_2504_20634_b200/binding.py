@@ -41,6 +41,8 @@ def _load():
     vp, sz, i, u64, f = ctypes.c_void_p, ctypes.c_size_t, ctypes.c_int, ctypes.c_uint64, ctypes.c_float
     L.fbsr_round.argtypes = [vp, vp, sz, i, i, i, u64, u64, f, vp]
     L.fbsr_round_bits.argtypes = [vp, vp, sz, i, i, i, vp, f, vp]
+    L.fbsr_round_mx.argtypes = [vp, vp, vp, sz, i, i, i, u64, u64, vp]
+    L.fbsr_round_mx.restype = i
     L.fbsr_round_lp.argtypes = [vp, i, vp, sz, i, i, i, u64, u64, f, vp]
     L.fbsr_round_lp.restype = i
     L.fbsr_stats_workspace_bytes.argtypes = []
@@ -147,6 +149,17 @@ def fbsr_round(src, fmt, variant, k_bits, seed, offset=0, scale=1.0, out=None):
         _check(_L.fbsr_round(_dev(src, torch.float32, "src"), po, src.numel(), _fmt(fmt), _var(variant), k_bits,
                              seed, offset, scale, _stream(src)), "fbsr_round")
     return out
+
+
+def fbsr_round_mx(src, fmt, variant, k_bits, seed, offset=0, out=None, scales=None):
+    """Block-scaled rounding (blocks of 32 elements, shared power-of-two scale); returns (codes, scale bytes)."""
+    out, po = _out(src, fmt, out)
+    if scales is None:
+        scales = torch.empty((src.numel() + 31) // 32, dtype=torch.uint8, device=src.device)
+    with torch.cuda.device(src.device):
+        _check(_L.fbsr_round_mx(_dev(src, torch.float32, "src"), po, _dev(scales, torch.uint8, "scales"), src.numel(),
+                                _fmt(fmt), _var(variant), k_bits, seed, offset, _stream(src)), "fbsr_round_mx")
+    return out, scales
 
 
 def fbsr_round_lp(src_codes, src_fmt, fmt, variant, k_bits, seed, offset=0, scale=1.0, out=None):

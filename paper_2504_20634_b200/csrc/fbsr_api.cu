@@ -88,6 +88,19 @@ int fbsr_round_lp(const void* src, int src_fmt, void* dst, size_t n, int dst_fmt
     return finish(dst_fmt == FBSR_E4M3 ? dispatch_lp_2(a) : dispatch_lp_3(a));
 }
 
+int fbsr_round_mx(const float* src, void* dst, uint8_t* scales, size_t n, int fmt, int variant, int k_bits,
+                  uint64_t seed, uint64_t offset, void* cuda_stream)
+{
+    const int ovf_ieee = take_overflow_flag(fmt);
+    if (int rc = check_round(src, dst, n, fmt, variant, k_bits, 1.0f)) return rc;
+    if (n > 0 && scales == nullptr) return FBSR_ERR_INVALID_ARG;
+    if (n == 0) return FBSR_OK;
+    CallArgs a = base_args(OP_ROUND_MX, variant, k_bits, n, seed, offset, dst, cuda_stream);
+    a.ovf_ieee = ovf_ieee;
+    a.src = src; a.scales = scales;
+    return finish(kRound[fmt](a));
+}
+
 int fbsr_round_bits(const float* src, void* dst, size_t n, int fmt, int variant, int k_bits,
                     const uint32_t* rand_words, float scale, void* cuda_stream)
 {

@@ -39,6 +39,8 @@ inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_
     o.u += h; o.w_lp = static_cast<const char*>(o.w_lp) + h * CODE_BYTES; return o;
 }
 
+[[maybe_unused]] inline bool op_aligned(const MxOp<FMT>& o, size_t h) { return aligned(o.src + h, 32) && h % 32 == 0; }
+[[maybe_unused]] inline MxOp<FMT> op_advance(MxOp<FMT> o, size_t h) { o.src += h; o.scales += h / 32; o.n -= h; return o; }
 template <int UF> inline bool op_aligned(const QatOp<FMT == E4M3 || FMT == E5M2 ? FMT : E4M3, UF>& o, size_t h)
 {
     return aligned(static_cast<const uint16_t*>(o.u16) + h, 16);      // w8 is checked as dst
@@ -184,6 +186,7 @@ int FBSR_CAT(dispatch_round_, FBSR_FMT)(const CallArgs& a)
     switch (a.op) {
     case OP_ROUND: return by_variant_and_k<RoundOp, false>(op, a);
     case OP_ROUND_BITS: return by_variant_and_k<RoundOp, true>(op, a);
+    case OP_ROUND_MX: return by_variant_and_k<MxOp<FMT>, false>(MxOp<FMT>{a.src, a.scales, a.n}, a);
     case OP_ROUND_STATS: {
         // Whole rows of 256 elements go to the row kernel when the pointers allow vector access, the rest to
         // the general kernel; each CTA leaves one partial in the workspace and they are summed in a fixed order.

@@ -6,7 +6,7 @@
 
 namespace fbsr {
 
-enum OpKind { OP_ROUND = 0, OP_ROUND_BITS, OP_ROUND_STATS, OP_SGD, OP_ADAM, OP_ACCUM, OP_ROUND_LP, OP_QAT };
+enum OpKind { OP_ROUND = 0, OP_ROUND_BITS, OP_ROUND_STATS, OP_SGD, OP_ADAM, OP_ACCUM, OP_ROUND_LP, OP_QAT, OP_ROUND_MX };
 
 // Everything an entry point hands to the per-format dispatcher.  Validated by the caller.
 struct CallArgs {
@@ -21,6 +21,7 @@ struct CallArgs {
     const float* src;
     float scale;
     const uint32_t* words;          // OP_ROUND_BITS
+    uint8_t* scales;                // OP_ROUND_MX: one exponent byte per block of 32
     const void* src_lp;             // OP_ROUND_LP: codes of src_fmt; OP_QAT: the 16-bit updates
     int src_fmt;
     // OP_ROUND_STATS

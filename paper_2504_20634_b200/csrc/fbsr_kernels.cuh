@@ -153,6 +153,62 @@ struct RoundOp {
     __device__ __forceinline__ uint32_t scalar(size_t i) const { return scaled_bits(src[i], scale); }
 };
 
+// Block-scaled rounding: 32 consecutive elements (4 lanes of a row) share a power-of-two scale taken from
+// their largest finite magnitude; the scale byte is written by the first lane of the block.
+template <int FMT>
+struct MxOp {
+    static constexpr int BATCH = ROW_BATCH, MIN_CTAS = FBSR_MIN_CTAS_ROUND;
+    static constexpr int EMAX = (int)(Format<FMT>::MAXBITS >> 23) - 127;        // floor(log2 M)
+    const float* src; uint8_t* scales; size_t n;
+    struct Regs { F8 x; };
+    __device__ __forceinline__ static int block_exponent(uint32_t amax_bits)
+    {
+        const int e = (int)(amax_bits >> 23) - 127 - EMAX;                       // subnormal or zero amax clamps to -127
+        return max(-127, min(127, e));
+    }
+    __device__ __forceinline__ static float inverse_scale(int e_blk)
+    {
+        const uint32_t field = (uint32_t)(127 - e_blk);                          // 0..254; 0 means 2^-127, a subnormal
+        return __uint_as_float(field ? field << 23 : 0x00400000u);
+    }
+    __device__ __forceinline__ static uint32_t finite_magnitude(float v)
+    {
+        const uint32_t m = __float_as_uint(v) & 0x7FFFFFFFu;
+        return m < 0x7F800000u ? m : 0u;
+    }
+    __device__ __forceinline__ void fetch(size_t elem, Regs& r) const { r.x = load_f8_stream(src + elem); }
+    __device__ __forceinline__ void finish(size_t elem, const Regs& r, float (&y)[8]) const
+    {
+        float x[8];
+        unpack(r.x, x);
+        uint32_t m = 0u;
+#pragma unroll
+        for (int c = 0; c < 8; ++c) m = max(m, finite_magnitude(x[c]));
+        m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, 1));
+        m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, 2));
+        const int e_blk = block_exponent(m);
+        const float s = inverse_scale(e_blk);
+#pragma unroll
+        for (int c = 0; c < 8; ++c) y[c] = __fmul_rn(x[c], s);
+        if ((threadIdx.x & 3) == 0) scales[elem / 32] = (uint8_t)(e_blk + 127);
+    }
+    __device__ __forceinline__ uint32_t exact_bits(const Regs& r, int c, float y) const
+    {
+        float x[8];
+        unpack(r.x, x);
+        return y != y ? __float_as_uint(x[c]) : __float_as_uint(y);
+    }
+    __device__ __forceinline__ uint32_t scalar(size_t i) const
+    {
+        const size_t b0 = i / 32 * 32, b1 = b0 + 32 < n ? b0 + 32 : n;
+        uint32_t m = 0u;
+        for (size_t j = b0; j < b1; ++j) m = max(m, finite_magnitude(src[j]));
+        const int e_blk = block_exponent(m);
+        if (i == b0) scales[i / 32] = (uint8_t)(e_blk + 127);
+        return scaled_bits(src[i], inverse_scale(e_blk));
+    }
+};
+
 // Source already in a 16-bit format: widen exactly (Eq. (1)), then scale.
 template <int SRC>
 struct LpSrcOp {

@@ -17,7 +17,7 @@ from paper_2504_20634_b200 import workloads
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--op", default="round", choices=["round", "sgd", "adam", "accumulate", "stats", "bits", "lp"])
+    ap.add_argument("--op", default="round", choices=["round", "sgd", "adam", "accumulate", "stats", "bits", "lp", "mx"])
     ap.add_argument("--src-fmt", default="bf16", help="source format for --op lp")
     ap.add_argument("--fmt", default="bf16")
     ap.add_argument("--variant", default="srf")
@@ -39,6 +39,10 @@ def main():
         codes = workloads.lp_sweep(n, args.src_fmt, device=dev)
         bytes_per_elem = 2 + code_bytes
         run = lambda s: fbsr.fbsr_round_lp(codes, args.src_fmt, args.fmt, args.variant, args.k, seed=1234, out=out)
+    elif args.op == "mx":
+        scales = torch.empty((n + 31) // 32, dtype=torch.uint8, device=dev)
+        bytes_per_elem = 4 + code_bytes + 1.0 / 32
+        run = lambda s: fbsr.fbsr_round_mx(x, args.fmt, args.variant, args.k, seed=1234, out=out, scales=scales)
     elif args.op == "bits":
         dpw = 32 // args.k
         words = torch.randint(0, 2 ** 31, ((n + dpw - 1) // dpw,), device=dev, dtype=torch.int32).view(torch.uint32)
