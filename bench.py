@@ -40,10 +40,10 @@ def sweep():
 
 
 # DRAM traffic of one 2^28-element bf16 launch, from the ncu capture summarised in
-# profiles/tile_kernel_round_bf16_srf_k4.txt (dram__bytes_read.sum + dram__bytes_write.sum of a 2^27-element
+# profiles/tile_kernel_round.txt (dram__bytes_read.sum + dram__bytes_write.sum of a 2^27-element
 # launch, scaled by the elements processed).  Valid only for the kernel sources it was taken from.
-TRAFFIC_BYTES_PER_LAUNCH = 2 * (536.895744e6 + 222.235136e6)
-TRAFFIC_KERNEL_SHA = "a8b81eeb66333071"
+TRAFFIC_BYTES_PER_LAUNCH = 2 * (536.891904e6 + 221.806080e6)
+TRAFFIC_KERNEL_SHA = "4c6d710406bdd5af"
 
 
 def kernel_source_sha():
