@@ -186,8 +186,9 @@ template <int K> struct Draws8 {
         return (b <= POS ? (w << (POS - b)) : (w >> (b - POS))) & (MASK << POS);
     }
 
-    // acc + (field of element c moved to bit POS).  The field is masked where it sits and the move
-    // is folded into a multiply-add, which runs on the FMA pipe instead of the busier integer pipe.
+    // acc + (field of element c moved to bit POS).  The field is masked where it sits; the move is written
+    // as a multiply by a power of two so that the compiler may fold it with the addition (shift-add or
+    // multiply-add, its choice).
     template <int POS>
     __device__ __forceinline__ uint32_t add_at(const int c, const uint32_t acc) const
     {
