@@ -43,7 +43,7 @@ def sweep():
 # profiles/tile_kernel_round.txt (dram__bytes_read.sum + dram__bytes_write.sum of a 2^27-element
 # launch, scaled by the elements processed).  Valid only for the kernel sources it was taken from.
 TRAFFIC_BYTES_PER_LAUNCH = 2 * (536.891904e6 + 221.806080e6)
-TRAFFIC_KERNEL_SHA = "4c6d710406bdd5af"
+TRAFFIC_KERNEL_SHA = "ce87a9b962a06918"
 
 
 def kernel_source_sha():

@@ -65,13 +65,19 @@ template <int K> struct Tile {
 };
 
 // ---------------------------------------------------------------------------- vector memory access
+#ifndef FBSR_STORE
+#define FBSR_STORE __stcs          // streaming store: the codes are not read again by this kernel
+#endif
 struct F8 { float4 a, b; };
 
 __device__ __forceinline__ F8 load_f8_stream(const float* p)
 {
     // 256-bit read-only load that does not allocate in L1: the data is used once.
     F8 v;
-    asm volatile("ld.global.nc.L1::no_allocate.L2::evict_first.v8.f32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+#ifndef FBSR_STREAM_LOAD
+#define FBSR_STREAM_LOAD "ld.global.nc.L1::no_allocate.L2::evict_first.v8.f32"
+#endif
+    asm volatile(FBSR_STREAM_LOAD " {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
                  : "=f"(v.a.x), "=f"(v.a.y), "=f"(v.a.z), "=f"(v.a.w),
                    "=f"(v.b.x), "=f"(v.b.y), "=f"(v.b.z), "=f"(v.b.w)
                  : "l"(p));
@@ -108,12 +114,12 @@ __device__ __forceinline__ void store_codes8(void* dst, size_t elem, const uint3
         uint4 v;
         v.x = c[0] | (c[1] << 16); v.y = c[2] | (c[3] << 16);
         v.z = c[4] | (c[5] << 16); v.w = c[6] | (c[7] << 16);
-        __stcs(reinterpret_cast<uint4*>(static_cast<uint16_t*>(dst) + elem), v);
+        FBSR_STORE(reinterpret_cast<uint4*>(static_cast<uint16_t*>(dst) + elem), v);
     } else {
         uint2 v;
         v.x = c[0] | (c[1] << 8) | (c[2] << 16) | (c[3] << 24);
         v.y = c[4] | (c[5] << 8) | (c[6] << 16) | (c[7] << 24);
-        __stcs(reinterpret_cast<uint2*>(static_cast<uint8_t*>(dst) + elem), v);
+        FBSR_STORE(reinterpret_cast<uint2*>(static_cast<uint8_t*>(dst) + elem), v);
     }
 }
 
@@ -448,7 +454,7 @@ __device__ __forceinline__ void store_row_fast(void* dst, size_t elem, const uin
         uint4 v;
         v.x = __byte_perm(t[0], t[1], 0x7632); v.y = __byte_perm(t[2], t[3], 0x7632);
         v.z = __byte_perm(t[4], t[5], 0x7632); v.w = __byte_perm(t[6], t[7], 0x7632);
-        __stcs(reinterpret_cast<uint4*>(static_cast<uint16_t*>(dst) + elem), v);
+        FBSR_STORE(reinterpret_cast<uint4*>(static_cast<uint16_t*>(dst) + elem), v);
     } else if constexpr (Format<FMT>::K == 16) {
         uint32_t o[4];
 #pragma unroll
@@ -456,7 +462,7 @@ __device__ __forceinline__ void store_row_fast(void* dst, size_t elem, const uin
             const uint32_t signs = __byte_perm(__float_as_uint(y[2 * j]), __float_as_uint(y[2 * j + 1]), 0x7632);
             o[j] = (t[2 * j] + t[2 * j + 1] * 65536u) | (signs & 0x80008000u);
         }
-        __stcs(reinterpret_cast<uint4*>(static_cast<uint16_t*>(dst) + elem), make_uint4(o[0], o[1], o[2], o[3]));
+        FBSR_STORE(reinterpret_cast<uint4*>(static_cast<uint16_t*>(dst) + elem), make_uint4(o[0], o[1], o[2], o[3]));
     } else {
         uint32_t o[2];
 #pragma unroll
@@ -467,7 +473,7 @@ __device__ __forceinline__ void store_row_fast(void* dst, size_t elem, const uin
             o[j] = (t[4 * j] + t[4 * j + 1] * 256u + t[4 * j + 2] * 65536u + t[4 * j + 3] * 16777216u) |
                    (signs & 0x80808080u);
         }
-        __stcs(reinterpret_cast<uint2*>(static_cast<uint8_t*>(dst) + elem), make_uint2(o[0], o[1]));
+        FBSR_STORE(reinterpret_cast<uint2*>(static_cast<uint8_t*>(dst) + elem), make_uint2(o[0], o[1]));
     }
 }
 
