@@ -298,7 +298,7 @@ __device__ __forceinline__ bool round_row_fast(const float (&y)[8], const Draws8
             if constexpr (VAR == SRFF) lo = (__float2uint_rz(steps) + d.template at<0>(c)) >> N;
             else if constexpr (VAR == SRF) lo = (__float2uint_rz(steps) + ((d.template at<0>(c) << 1) | 1u)) >> (N + 1);
             else lo = (__float2uint_rn(steps) + d.template at<0>(c)) >> N;
-            t[c] = a < min_normal ? lo : hi;
+            t[c] = (a < min_normal ? lo : hi) << (32 - F::K);        // code in the top K bits, like the one-regime form
         }
         return flag != flag;
     } else {
@@ -319,22 +319,27 @@ __device__ __forceinline__ bool round_row_fast(const float (&y)[8], const Draws8
             }
             flag = __fmaf_rn(y[c], 0.0f, flag);               // NaN iff y is Inf or NaN
         }
+        // Other formats: saturate the pattern first (what is added below stays under one code step), then move
+        // it left by L so that the code ends at bit 30: packing then takes whole bytes and needs no shift.
+        constexpr int L = FMT == BF16 ? 0 : 31 - (F::K - 1) - SH0;
+        if constexpr (FMT != BF16) u = min(u, F::MAXCODE << SH0);
+        const uint32_t base = u * (1u << L);
+        const uint32_t floor_lsb = ((u >> POS) & 1u) << L;     // used by the nearest-even / nearest-odd forms only
+        constexpr uint32_t HALF = POS > 0 ? 1u << (POS > 0 ? POS - 1 + L : 0) : 0u;
+        constexpr uint32_t BELOW_HALF = POS > 0 ? ((1u << (POS > 0 ? POS - 1 : 0)) - 1u) << L : 0u;
         uint32_t sum;
         if constexpr (EFF == RTA) {
-            sum = u + (1u << (POS - 1));                      // ties away: add half a step
+            sum = base + HALF;                                // ties away: add half a step
         } else if constexpr (EFF == RTNE || EFF == RTO) {
-            const uint32_t floor_lsb = (u >> POS) & 1u;
-            sum = u + ((1u << (POS - 1)) - 1u) + (EFF == RTNE ? floor_lsb : floor_lsb ^ 1u);
+            sum = base + BELOW_HALF + (EFF == RTNE ? floor_lsb : floor_lsb ^ (1u << L));
         } else if constexpr (EFF == SRFF) {
-            sum = d.template add_at<POS>(c, u);
+            sum = d.template add_at<POS + L>(c, base);
         } else if constexpr (EFF == SRF) {
-            sum = d.template add_at<POS>(c, u + (1u << (POS - 1)));
+            sum = d.template add_at<POS + L>(c, base + HALF);
         } else {
-            const uint32_t lsb = (u >> POS) & 1u;
-            sum = d.template add_at<POS>(c, u + ((1u << (POS - 1)) - 1u) + lsb);
+            sum = d.template add_at<POS + L>(c, base + BELOW_HALF + floor_lsb);
         }
-        if constexpr (FMT == BF16) t[c] = sum;                // code = bits 16..31
-        else t[c] = min(sum >> SH0, F::MAXCODE);
+        t[c] = sum;                                           // code in the top K bits (bf16: with its sign)
     }
     return flag != flag;
     }

@@ -445,8 +445,8 @@ struct QatOp {
 };
 
 // ---------------------------------------------------------------------------- packing a row of codes
-// Fast rows: t[] as left by round_row_fast (bfloat16: code in bits 16..31 with the sign;
-// other formats: magnitude code, sign still to be taken from y).
+// Fast rows: t[] as left by round_row_fast: the code sits in the top K bits of each word (bfloat16 with its sign,
+// the other formats with bit 31 clear and the sign still to be taken from y), so packing is byte selection.
 template <int FMT>
 __device__ __forceinline__ void store_row_fast(void* dst, size_t elem, const uint32_t (&t)[8], const float (&y)[8])
 {
@@ -459,19 +459,20 @@ __device__ __forceinline__ void store_row_fast(void* dst, size_t elem, const uin
         uint32_t o[4];
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
+            const uint32_t codes = __byte_perm(t[2 * j], t[2 * j + 1], 0x7632);
             const uint32_t signs = __byte_perm(__float_as_uint(y[2 * j]), __float_as_uint(y[2 * j + 1]), 0x7632);
-            o[j] = (t[2 * j] + t[2 * j + 1] * 65536u) | (signs & 0x80008000u);
+            o[j] = codes | (signs & 0x80008000u);
         }
         FBSR_STORE(reinterpret_cast<uint4*>(static_cast<uint16_t*>(dst) + elem), make_uint4(o[0], o[1], o[2], o[3]));
     } else {
         uint32_t o[2];
 #pragma unroll
         for (int j = 0; j < 2; ++j) {
+            const uint32_t c01 = __byte_perm(t[4 * j], t[4 * j + 1], 0x7373);
+            const uint32_t c23 = __byte_perm(t[4 * j + 2], t[4 * j + 3], 0x7373);
             const uint32_t s01 = __byte_perm(__float_as_uint(y[4 * j]), __float_as_uint(y[4 * j + 1]), 0x7373);
             const uint32_t s23 = __byte_perm(__float_as_uint(y[4 * j + 2]), __float_as_uint(y[4 * j + 3]), 0x7373);
-            const uint32_t signs = __byte_perm(s01, s23, 0x5410);
-            o[j] = (t[4 * j] + t[4 * j + 1] * 256u + t[4 * j + 2] * 65536u + t[4 * j + 3] * 16777216u) |
-                   (signs & 0x80808080u);
+            o[j] = __byte_perm(c01, c23, 0x5410) | (__byte_perm(s01, s23, 0x5410) & 0x80808080u);
         }
         FBSR_STORE(reinterpret_cast<uint2*>(static_cast<uint8_t*>(dst) + elem), make_uint2(o[0], o[1]));
     }
