@@ -234,7 +234,7 @@ int fbsr_round_host(const float* src_host, void* dst_host, size_t n, int fmt, in
                     uint64_t seed, uint64_t offset, float scale, void* dev_workspace,
                     size_t workspace_bytes, void* cuda_stream);
 
-/* Elements per warp tile of the fast path for k_bits: `offset` values that are
+/* A common multiple of the warp-tile sizes the entry points use for k_bits: `offset` values that are
  * multiples of it keep a sharded call on the fast path.  0 if k_bits is invalid. */
 size_t fbsr_tile_elements(int k_bits);
 

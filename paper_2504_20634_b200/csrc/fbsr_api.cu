@@ -257,8 +257,7 @@ size_t fbsr_tile_elements(int k_bits)
     const int dpw = 32 / k_bits;
     if ((dpw & (dpw - 1)) == 0) return 1024;                 // power-of-two draws per word: 4 rows
     const int r0 = (dpw % 2 == 0) ? dpw / 2 : dpw;           // rows that hold whole generator calls
-    const int rows = r0 >= 4 ? r0 : r0 * ((4 + r0 - 1) / r0);
-    return (size_t)rows * 256;
+    return (size_t)(r0 % 2 == 0 ? r0 : 2 * r0) * 256;        // an even number of them
 }
 
 size_t fbsr_round_host_min_workspace(void) { return (size_t)1 << 20; }

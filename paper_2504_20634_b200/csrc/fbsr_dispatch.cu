@@ -43,7 +43,7 @@ inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_
 [[maybe_unused]] inline MxOp<FMT> op_advance(MxOp<FMT> o, size_t h) { o.src += h; o.scales += h / 32; o.n -= h; return o; }
 template <int UF> inline bool op_aligned(const QatOp<FMT == E4M3 || FMT == E5M2 ? FMT : E4M3, UF>& o, size_t h)
 {
-    return aligned(static_cast<const uint16_t*>(o.u16) + h, 16);      // w8 is checked as dst
+    return aligned(static_cast<const uint16_t*>(o.u16) + h, 32);      // w8 is checked as dst
 }
 template <int UF> inline QatOp<FMT == E4M3 || FMT == E5M2 ? FMT : E4M3, UF> op_advance(QatOp<FMT == E4M3 || FMT == E5M2 ? FMT : E4M3, UF> o, size_t h)
 {
@@ -51,7 +51,7 @@ template <int UF> inline QatOp<FMT == E4M3 || FMT == E5M2 ? FMT : E4M3, UF> op_a
 }
 template <int SRC> inline bool op_aligned(const LpSrcOp<SRC>& o, size_t h)
 {
-    return aligned(static_cast<const uint16_t*>(o.src) + h, 16);
+    return aligned(static_cast<const uint16_t*>(o.src) + h, 32);
 }
 template <int SRC> inline LpSrcOp<SRC> op_advance(LpSrcOp<SRC> o, size_t h)
 {
@@ -63,7 +63,7 @@ struct Plan { size_t head, n_tiles, tail_begin; };
 template <class Op, int VAR, int K, bool BITS>
 int launch_tiles(const Op& op, const CallArgs& a, const Plan& p)
 {
-    using T = Tile<K>;
+    using T = Tile<K, Op::OCTETS>;
     auto kern = tile_kernel<Op, FMT, VAR, K, BITS>;
     // One tile per warp, CTAs handed out by the hardware scheduler.  A persistent grid with a static
     // tile stride measured 5-10 % slower here: multiprocessors do not all see the same memory
@@ -105,11 +105,11 @@ int launch_generic(const Op& op, const CallArgs& a, size_t i_begin, size_t i_end
 template <class Op, int K, bool BITS>
 Plan make_plan(const Op& op, const CallArgs& a)
 {
-    using T = Tile<K>;
+    using T = Tile<K, Op::OCTETS>;
     Plan p{0, 0, 0};
     const uint64_t off = BITS ? 0 : a.offset;
     const size_t head = (size_t)((T::ELEMS - off % T::ELEMS) % T::ELEMS);
-    const size_t dst_align = CODE_BYTES == 2 ? 16 : 8;
+    const size_t dst_align = (CODE_BYTES == 2 ? 16 : 8) * Op::OCTETS;      // one vector store per lane-row
     if (head < a.n && op_aligned(op, head) &&
         aligned(static_cast<char*>(a.dst) + head * CODE_BYTES, dst_align)) {
         p.head = head;

@@ -49,15 +49,16 @@ constexpr int ROW_BATCH = FBSR_ROW_BATCH;
 constexpr int CTA_THREADS = WARPS_PER_CTA * 32;
 constexpr int ROW_ELEMS = 256;          // 32 lanes x 8 elements
 
-template <int K> struct Tile {
+template <int K, int OCT = 1> struct Tile {
     static constexpr int DPW = 32 / K;                        // draws per word
     static constexpr int E = 4 * DPW;                         // elements per Philox call
     static constexpr bool POW2 = (DPW & (DPW - 1)) == 0;
-    // Power-of-two dpw: 4 rows (1024 elements) always hold whole calls.  Otherwise the smallest
-    // number of rows that does (dpw rows, or dpw/2 when dpw is even), doubled while below 4.
+    // Power-of-two dpw: 4 lane-rows of 256 elements (1024) always hold whole calls.  Otherwise the smallest
+    // number of them that does (dpw, or dpw/2 when dpw is even), doubled while below 4; and doubled once more
+    // if an op that takes OCT octets per lane could not split it into whole rows of 256 * OCT elements.
     static constexpr int R0 = (DPW % 2 == 0) ? DPW / 2 : DPW;
-    static constexpr int ROWS = POW2 ? 4 : (R0 >= 4 ? R0 : R0 * ((4 + R0 - 1) / R0));
-    static constexpr int ELEMS = ROWS * ROW_ELEMS;
+    static constexpr int ROWS1 = POW2 ? 4 : (R0 >= 4 ? R0 : R0 * ((4 + R0 - 1) / R0));
+    static constexpr int ELEMS = ROWS1 * ROW_ELEMS * (ROWS1 % OCT == 0 ? 1 : 2);
     static constexpr int CALLS = ELEMS / E;                   // Philox calls per tile
     static constexpr int WORDS = ELEMS / DPW;                 // random words per tile
     static constexpr uint32_t MASK = (1u << K) - 1u;
@@ -107,20 +108,43 @@ __device__ __forceinline__ void unpack(const F8& v, float (&x)[8])
     x[4] = v.b.x; x[5] = v.b.y; x[6] = v.b.z; x[7] = v.b.w;
 }
 
+// Words that 8 packed codes occupy.
+template <int FMT> struct WordsPerOctet { static constexpr int value = Format<FMT>::K == 16 ? 4 : 2; };
+
+// 8 plain codes -> packed words.
+template <int FMT>
+__device__ __forceinline__ void pack_codes8(const uint32_t (&c)[8], uint32_t* out)
+{
+    if constexpr (Format<FMT>::K == 16) {
+        out[0] = c[0] | (c[1] << 16); out[1] = c[2] | (c[3] << 16);
+        out[2] = c[4] | (c[5] << 16); out[3] = c[6] | (c[7] << 16);
+    } else {
+        out[0] = c[0] | (c[1] << 8) | (c[2] << 16) | (c[3] << 24);
+        out[1] = c[4] | (c[5] << 8) | (c[6] << 16) | (c[7] << 24);
+    }
+}
+
+// N packed words -> one streaming vector store (8, 16 or 32 bytes).
+template <int NWORDS>
+__device__ __forceinline__ void store_words(void* p, const uint32_t (&w)[NWORDS])
+{
+    static_assert(NWORDS == 2 || NWORDS == 4 || NWORDS == 8, "8-, 16- or 32-byte stores");
+    if constexpr (NWORDS == 2) {
+        FBSR_STORE(reinterpret_cast<uint2*>(p), make_uint2(w[0], w[1]));
+    } else if constexpr (NWORDS == 4) {
+        FBSR_STORE(reinterpret_cast<uint4*>(p), make_uint4(w[0], w[1], w[2], w[3]));
+    } else {
+        FBSR_STORE(reinterpret_cast<uint4*>(p), make_uint4(w[0], w[1], w[2], w[3]));
+        FBSR_STORE(reinterpret_cast<uint4*>(p) + 1, make_uint4(w[4], w[5], w[6], w[7]));
+    }
+}
+
 template <int FMT>
 __device__ __forceinline__ void store_codes8(void* dst, size_t elem, const uint32_t (&c)[8])
 {
-    if constexpr (Format<FMT>::K == 16) {
-        uint4 v;
-        v.x = c[0] | (c[1] << 16); v.y = c[2] | (c[3] << 16);
-        v.z = c[4] | (c[5] << 16); v.w = c[6] | (c[7] << 16);
-        FBSR_STORE(reinterpret_cast<uint4*>(static_cast<uint16_t*>(dst) + elem), v);
-    } else {
-        uint2 v;
-        v.x = c[0] | (c[1] << 8) | (c[2] << 16) | (c[3] << 24);
-        v.y = c[4] | (c[5] << 8) | (c[6] << 16) | (c[7] << 24);
-        FBSR_STORE(reinterpret_cast<uint2*>(static_cast<uint8_t*>(dst) + elem), v);
-    }
+    uint32_t w[WordsPerOctet<FMT>::value];
+    pack_codes8<FMT>(c, w);
+    store_words<WordsPerOctet<FMT>::value>(static_cast<char*>(dst) + elem * (Format<FMT>::K / 8), w);
 }
 
 template <int FMT>
@@ -138,7 +162,7 @@ __device__ __forceinline__ void store_code1(void* dst, size_t elem, uint32_t c)
 // scalar(): the same for one element on the slow path.
 
 struct RoundOp {
-    static constexpr int BATCH = ROW_BATCH, MIN_CTAS = FBSR_MIN_CTAS_ROUND;
+    static constexpr int BATCH = ROW_BATCH, MIN_CTAS = FBSR_MIN_CTAS_ROUND, OCTETS = 1;
     const float* src;
     float scale;
     struct Regs { F8 x; };
@@ -163,7 +187,7 @@ struct RoundOp {
 // their largest finite magnitude; the scale byte is written by the first lane of the block.
 template <int FMT>
 struct MxOp {
-    static constexpr int BATCH = ROW_BATCH, MIN_CTAS = FBSR_MIN_CTAS_ROUND;
+    static constexpr int BATCH = ROW_BATCH, MIN_CTAS = FBSR_MIN_CTAS_ROUND, OCTETS = 1;
     static constexpr int EMAX = (int)(Format<FMT>::MAXBITS >> 23) - 127;        // floor(log2 M)
     const float* src; uint8_t* scales; size_t n;
     struct Regs { F8 x; };
@@ -219,41 +243,35 @@ struct MxOp {
 template <int SRC>
 struct LpSrcOp {
     static_assert(SRC == BF16 || SRC == FP16, "16-bit sources");
-    static constexpr int BATCH = ROW_BATCH, MIN_CTAS = FBSR_MIN_CTAS_ROUND;
+    // two octets per lane: one 256-bit load of 16 codes, one 128-bit store of 16 eight-bit codes
+    static constexpr int BATCH = ROW_BATCH, MIN_CTAS = FBSR_MIN_CTAS_ROUND, OCTETS = 2;
     const void* src;
     float scale;
-    struct Regs { uint4 c; };
-    __device__ __forceinline__ static float widen(uint32_t code)
-    {
-        if constexpr (SRC == BF16) return __uint_as_float(code << 16);
-        else return __half2float(__ushort_as_half((unsigned short)code));
-    }
+    struct Regs { uint32_t c[8]; };
     __device__ __forceinline__ void fetch(size_t elem, Regs& r) const
     {
-        const uint4* p = reinterpret_cast<const uint4*>(static_cast<const uint16_t*>(src) + elem);
-        asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
-                     : "=r"(r.c.x), "=r"(r.c.y), "=r"(r.c.z), "=r"(r.c.w) : "l"(p));
+        const uint16_t* p = static_cast<const uint16_t*>(src) + elem;
+        asm volatile("ld.global.nc.L1::no_allocate.L2::evict_first.v8.u32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                     : "=r"(r.c[0]), "=r"(r.c[1]), "=r"(r.c[2]), "=r"(r.c[3]),
+                       "=r"(r.c[4]), "=r"(r.c[5]), "=r"(r.c[6]), "=r"(r.c[7]) : "l"(p));
     }
-    __device__ __forceinline__ uint32_t code_of(const Regs& r, int c) const
+    __device__ __forceinline__ void finish(size_t, const Regs& r, int o, float (&y)[8]) const
     {
-        const uint32_t w = c < 2 ? r.c.x : c < 4 ? r.c.y : c < 6 ? r.c.z : r.c.w;
-        return (c & 1) ? (w >> 16) : (w & 0xFFFFu);
-    }
-    __device__ __forceinline__ void finish(size_t, const Regs& r, float (&y)[8]) const
-    {
-        const uint32_t cw[4] = {r.c.x, r.c.y, r.c.z, r.c.w};
 #pragma unroll
         for (int c = 0; c < 8; ++c) {
+            const uint32_t w = r.c[4 * o + (c >> 1)];
             float v;
-            if constexpr (SRC == BF16) v = __uint_as_float((c & 1) ? (cw[c >> 1] & 0xFFFF0000u) : (cw[c >> 1] << 16));
-            else v = widen((c & 1) ? (cw[c >> 1] >> 16) : (cw[c >> 1] & 0xFFFFu));
+            if constexpr (SRC == BF16) v = __uint_as_float((c & 1) ? (w & 0xFFFF0000u) : (w << 16));
+            else v = __half2float(__ushort_as_half((unsigned short)((c & 1) ? (w >> 16) : (w & 0xFFFFu))));
             y[c] = __fmul_rn(v, scale);
         }
     }
-    __device__ __forceinline__ uint32_t exact_bits(const Regs& r, int c, float y) const
+    __device__ __forceinline__ uint32_t exact_bits(const Regs& r, int o, int c, float y) const
     {
         // a NaN keeps the sign of the stored code
-        return y != y ? __float_as_uint(decode_element<SRC>(code_of(r, c))) : __float_as_uint(y);
+        const uint32_t w = r.c[4 * o + (c >> 1)];
+        const uint32_t code = (c & 1) ? (w >> 16) : (w & 0xFFFFu);
+        return y != y ? __float_as_uint(decode_element<SRC>(code)) : __float_as_uint(y);
     }
     __device__ __forceinline__ uint32_t scalar(size_t i) const
     {
@@ -264,7 +282,7 @@ struct LpSrcOp {
 
 // m' = fma(mu, m, g);  w' = fma(-lr, m', w)
 struct SgdOp {
-    static constexpr int BATCH = ROW_BATCH >= 2 ? ROW_BATCH / 2 : 1, MIN_CTAS = FBSR_MIN_CTAS_SGD;
+    static constexpr int BATCH = ROW_BATCH >= 2 ? ROW_BATCH / 2 : 1, MIN_CTAS = FBSR_MIN_CTAS_SGD, OCTETS = 1;
     float* w; const float* g; float* m;
     float neg_lr, mu;
     struct Regs { F8 w, g, m; };
@@ -297,7 +315,7 @@ struct SgdOp {
 
 // m' = fma(b1, m, a1 g); v' = fma(b2, v, (a2 g) g); d = sqrt(v') c2 + eps; w' = fma(-c1, m'/d, w)
 struct AdamOp {
-    static constexpr int BATCH = ROW_BATCH >= 2 ? ROW_BATCH / 2 : 1, MIN_CTAS = FBSR_MIN_CTAS_ADAM;
+    static constexpr int BATCH = ROW_BATCH >= 2 ? ROW_BATCH / 2 : 1, MIN_CTAS = FBSR_MIN_CTAS_ADAM, OCTETS = 1;
     float* w; const float* g; float* m; float* v;
     float beta1, beta2, eps, neg_c1, c2, a1, a2;
     struct Regs { F8 w, g, m, v; };
@@ -354,7 +372,7 @@ __device__ __forceinline__ void decode4(uint32_t w, float (&v)[4])
 // y = fl32(value(w_lp) + u); the codes are rewritten in place by the caller of finish()
 template <int FMT>
 struct AccumOp {
-    static constexpr int BATCH = ROW_BATCH, MIN_CTAS = FBSR_MIN_CTAS_ROUND;
+    static constexpr int BATCH = ROW_BATCH, MIN_CTAS = FBSR_MIN_CTAS_ROUND, OCTETS = 1;
     const void* w_lp; const float* u;
     struct Regs { F8 u; uint4 c; };
     __device__ __forceinline__ void fetch(size_t elem, Regs& r) const
@@ -400,9 +418,10 @@ struct AccumOp {
 template <int WF, int UF>
 struct QatOp {
     static_assert((WF == E4M3 || WF == E5M2) && (UF == BF16 || UF == FP16), "8-bit weights, 16-bit updates");
-    static constexpr int BATCH = ROW_BATCH, MIN_CTAS = FBSR_MIN_CTAS_ROUND;
+    // two octets per lane: 16 weight codes (128 bits) and 16 update codes (256 bits) in, 16 weight codes out
+    static constexpr int BATCH = ROW_BATCH >= 2 ? ROW_BATCH / 2 : 1, MIN_CTAS = FBSR_MIN_CTAS_ROUND, OCTETS = 2;
     const void* w8; const void* u16;
-    struct Regs { uint2 w; uint4 u; };
+    struct Regs { uint32_t w[4]; uint32_t u[8]; };
     __device__ __forceinline__ static float sum16(uint32_t wcode, uint32_t ucode)
     {
         return sum16v(decode_element<WF>(wcode), ucode);
@@ -420,24 +439,25 @@ struct QatOp {
     }
     __device__ __forceinline__ void fetch(size_t elem, Regs& r) const
     {
-        r.w = *reinterpret_cast<const uint2*>(static_cast<const uint8_t*>(w8) + elem);
-        const uint4* p = reinterpret_cast<const uint4*>(static_cast<const uint16_t*>(u16) + elem);
-        asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
-                     : "=r"(r.u.x), "=r"(r.u.y), "=r"(r.u.z), "=r"(r.u.w) : "l"(p));
+        const uint4 w = *reinterpret_cast<const uint4*>(static_cast<const uint8_t*>(w8) + elem);
+        r.w[0] = w.x; r.w[1] = w.y; r.w[2] = w.z; r.w[3] = w.w;
+        const uint16_t* p = static_cast<const uint16_t*>(u16) + elem;
+        asm volatile("ld.global.nc.L1::no_allocate.L2::evict_first.v8.u32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                     : "=r"(r.u[0]), "=r"(r.u[1]), "=r"(r.u[2]), "=r"(r.u[3]),
+                       "=r"(r.u[4]), "=r"(r.u[5]), "=r"(r.u[6]), "=r"(r.u[7]) : "l"(p));
     }
-    __device__ __forceinline__ void finish(size_t, const Regs& r, float (&y)[8]) const
+    __device__ __forceinline__ void finish(size_t, const Regs& r, int o, float (&y)[8]) const
     {
-        const uint32_t uw[4] = {r.u.x, r.u.y, r.u.z, r.u.w};
         float lo[4], hi[4];
-        decode4<WF>(r.w.x, lo);
-        decode4<WF>(r.w.y, hi);
+        decode4<WF>(r.w[2 * o], lo);
+        decode4<WF>(r.w[2 * o + 1], hi);
 #pragma unroll
         for (int c = 0; c < 8; ++c) {
-            const uint32_t ucode = (uw[c >> 1] >> ((c & 1) * 16)) & 0xFFFFu;
+            const uint32_t ucode = (r.u[4 * o + (c >> 1)] >> ((c & 1) * 16)) & 0xFFFFu;
             y[c] = sum16v(c < 4 ? lo[c] : hi[c - 4], ucode);
         }
     }
-    __device__ __forceinline__ uint32_t exact_bits(const Regs&, int, float y) const { return arith_bits(y); }
+    __device__ __forceinline__ uint32_t exact_bits(const Regs&, int, int, float y) const { return arith_bits(y); }
     __device__ __forceinline__ uint32_t scalar(size_t i) const
     {
         return arith_bits(sum16(static_cast<const uint8_t*>(w8)[i], static_cast<const uint16_t*>(u16)[i]));
@@ -448,33 +468,27 @@ struct QatOp {
 // Fast rows: t[] as left by round_row_fast: the code sits in the top K bits of each word (bfloat16 with its sign,
 // the other formats with bit 31 clear and the sign still to be taken from y), so packing is byte selection.
 template <int FMT>
-__device__ __forceinline__ void store_row_fast(void* dst, size_t elem, const uint32_t (&t)[8], const float (&y)[8])
+__device__ __forceinline__ void pack_row_fast(const uint32_t (&t)[8], const float (&y)[8], uint32_t* out)
 {
     if constexpr (FMT == BF16) {
-        uint4 v;
-        v.x = __byte_perm(t[0], t[1], 0x7632); v.y = __byte_perm(t[2], t[3], 0x7632);
-        v.z = __byte_perm(t[4], t[5], 0x7632); v.w = __byte_perm(t[6], t[7], 0x7632);
-        FBSR_STORE(reinterpret_cast<uint4*>(static_cast<uint16_t*>(dst) + elem), v);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) out[j] = __byte_perm(t[2 * j], t[2 * j + 1], 0x7632);
     } else if constexpr (Format<FMT>::K == 16) {
-        uint32_t o[4];
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
             const uint32_t codes = __byte_perm(t[2 * j], t[2 * j + 1], 0x7632);
             const uint32_t signs = __byte_perm(__float_as_uint(y[2 * j]), __float_as_uint(y[2 * j + 1]), 0x7632);
-            o[j] = codes | (signs & 0x80008000u);
+            out[j] = codes | (signs & 0x80008000u);
         }
-        FBSR_STORE(reinterpret_cast<uint4*>(static_cast<uint16_t*>(dst) + elem), make_uint4(o[0], o[1], o[2], o[3]));
     } else {
-        uint32_t o[2];
 #pragma unroll
         for (int j = 0; j < 2; ++j) {
             const uint32_t c01 = __byte_perm(t[4 * j], t[4 * j + 1], 0x7373);
             const uint32_t c23 = __byte_perm(t[4 * j + 2], t[4 * j + 3], 0x7373);
             const uint32_t s01 = __byte_perm(__float_as_uint(y[4 * j]), __float_as_uint(y[4 * j + 1]), 0x7373);
             const uint32_t s23 = __byte_perm(__float_as_uint(y[4 * j + 2]), __float_as_uint(y[4 * j + 3]), 0x7373);
-            o[j] = __byte_perm(c01, c23, 0x5410) | (__byte_perm(s01, s23, 0x5410) & 0x80808080u);
+            out[j] = __byte_perm(c01, c23, 0x5410) | (__byte_perm(s01, s23, 0x5410) & 0x80808080u);
         }
-        FBSR_STORE(reinterpret_cast<uint2*>(static_cast<uint8_t*>(dst) + elem), make_uint2(o[0], o[1]));
     }
 }
 
@@ -488,7 +502,7 @@ __global__ void __launch_bounds__(CTA_THREADS, Op::MIN_CTAS)
 tile_kernel(const Op op, void* __restrict__ dst, const uint64_t n_tiles, const uint64_t call0,
             const uint32_t k0, const uint32_t k1, const uint32_t* __restrict__ words, const uint32_t tail_count)
 {
-    using T = Tile<K>;
+    using T = Tile<K, Op::OCTETS>;
     constexpr bool DRAWS = VAR < RTNE;                     // the deterministic modes use no random bits
     // The elements after the last whole tile (fewer than one tile) are done by CTA 0, one element per
     // thread and step, each with its own generator call: it starts first and overlaps the tiles.
@@ -522,6 +536,19 @@ tile_kernel(const Op op, void* __restrict__ dst, const uint64_t n_tiles, const u
         const size_t e0 = (size_t)tile * T::ELEMS;
         const uint64_t tile_call0 = call0 + tile * T::CALLS;
 
+        // A lane takes OCT octets (8 consecutive elements each) per row, so a row is 256 * OCT elements; rows are
+        // taken in equal batches of at most Op::BATCH (5 rows: 3 + 2, not 4 + 1).
+        constexpr int OCT = Op::OCTETS;
+        constexpr int ROW = ROW_ELEMS * OCT, ROWS = T::ELEMS / ROW;
+        static_assert(T::ELEMS % ROW == 0, "whole rows per tile");
+        constexpr int N_BATCHES = (ROWS + Op::BATCH - 1) / Op::BATCH;
+        constexpr int BATCH = (ROWS + N_BATCHES - 1) / N_BATCHES;
+        constexpr int WPO = WordsPerOctet<FMT>::value;
+        // The loads of the first batch of rows are issued before the generator calls, which then run in their shadow.
+        typename Op::Regs regs[BATCH];
+#pragma unroll
+        for (int j = 0; j < BATCH; ++j) op.fetch(e0 + j * ROW + lane * 8 * OCT, regs[j]);
+
         if constexpr (!DRAWS) {
         } else if constexpr (BITS) {
             const uint32_t* src_words = words + tile * T::WORDS;
@@ -539,41 +566,49 @@ tile_kernel(const Op op, void* __restrict__ dst, const uint64_t n_tiles, const u
             __syncwarp();
         }
 
-        // rows are taken in equal batches of at most Op::BATCH (5 rows: 3 + 2, not 4 + 1)
-        constexpr int N_BATCHES = (T::ROWS + Op::BATCH - 1) / Op::BATCH;
-        constexpr int BATCH = (T::ROWS + N_BATCHES - 1) / N_BATCHES;
 #pragma unroll
-        for (int rb = 0; rb < T::ROWS; rb += BATCH) {
-            typename Op::Regs regs[BATCH];
+        for (int rb = 0; rb < ROWS; rb += BATCH) {
+            if (rb > 0) {
 #pragma unroll
-            for (int j = 0; j < BATCH; ++j)
-                if (rb + j < T::ROWS) op.fetch(e0 + (rb + j) * ROW_ELEMS + lane * 8, regs[j]);
+                for (int j = 0; j < BATCH; ++j)
+                    if (rb + j < ROWS) op.fetch(e0 + (rb + j) * ROW + lane * 8 * OCT, regs[j]);
+            }
 #pragma unroll
             for (int j = 0; j < BATCH; ++j) {
-                if (rb + j < T::ROWS) {
-                    const int p0 = (rb + j) * ROW_ELEMS + lane * 8;
-                    float y[8];
-                    op.finish(e0 + p0, regs[j], y);
-                    Draws8<K> d;
-                    if constexpr (!DRAWS) {
-                    } else if constexpr (OWN_CALL) {
-                        d.from_call(philox_block(tile_call0 + (rb + j) * 32 + lane, k0, k1));
-                    } else {
-                        d.from_stream(wb, p0);
-                    }
-                    uint32_t t[8];
-                    const bool redo = round_row_fast<FMT, VAR, K>(y, d, t);
-                    if (!redo) {
-                        store_row_fast<FMT>(dst, e0 + p0, t, y);
-                    } else {
-                        // a special value somewhere in this lane's row (rare): element-wise, exact
-                        uint32_t c[8];
+                if (rb + j < ROWS) {
+                    const int p0 = (rb + j) * ROW + lane * 8 * OCT;
+                    uint32_t packed[OCT * WPO];
 #pragma unroll
-                        for (int i = 0; i < 8; ++i)
-                            c[i] = round_core<FMT, false>(op.exact_bits(regs[j], i, y[i]), d.template at<0>(i), VAR, K,
-                                                          nullptr);
-                        store_codes8<FMT>(dst, e0 + p0, c);
+                    for (int o = 0; o < OCT; ++o) {
+                        const int po = p0 + 8 * o;
+                        float y[8];
+                        if constexpr (OCT == 1) op.finish(e0 + po, regs[j], y);
+                        else op.finish(e0 + po, regs[j], o, y);
+                        Draws8<K> d;
+                        if constexpr (!DRAWS) {
+                        } else if constexpr (OWN_CALL) {
+                            d.from_call(philox_block(tile_call0 + po / 8, k0, k1));
+                        } else {
+                            d.from_stream(wb, po);
+                        }
+                        uint32_t t[8];
+                        const bool redo = round_row_fast<FMT, VAR, K>(y, d, t);
+                        if (!redo) {
+                            pack_row_fast<FMT>(t, y, packed + o * WPO);
+                        } else {
+                            // a special value somewhere in this octet (rare): element-wise, exact
+                            uint32_t c[8];
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) {
+                                uint32_t bits;
+                                if constexpr (OCT == 1) bits = op.exact_bits(regs[j], i, y[i]);
+                                else bits = op.exact_bits(regs[j], o, i, y[i]);
+                                c[i] = round_core<FMT, false>(bits, d.template at<0>(i), VAR, K, nullptr);
+                            }
+                            pack_codes8<FMT>(c, packed + o * WPO);
+                        }
                     }
+                    store_words<OCT * WPO>(static_cast<char*>(dst) + (e0 + p0) * (Format<FMT>::K / 8), packed);
                 }
             }
         }

@@ -14,8 +14,8 @@ def tile_elements(k_bits):
     if dpw & (dpw - 1) == 0:
         return 1024
     rows = dpw // 2 if dpw % 2 == 0 else dpw
-    if rows < 4:
-        rows *= -(-4 // rows)
+    if rows % 2:
+        rows *= 2
     return rows * 256
 
 
