@@ -15,13 +15,14 @@ _SRC = os.path.join(_HERE, "fbsr_oracle.c")
 _LIB = os.path.join(_HERE, "libfbsr_oracle.so")
 _CFLAGS = ["-O2", "-std=gnu11", "-ffp-contract=off", "-fno-fast-math", "-shared", "-fPIC"]
 
-FMT = {"bf16": 0, "fp16": 1, "e4m3": 2, "e5m2": 3}
+FMT = {"bf16": 0, "fp16": 1, "e4m3": 2, "e5m2": 3, "b8p4": 4}
 OVF_IEEE = 0x100                   # or-ed into a format id: paper-literal overflow instead of saturation
-for _name in ("bf16", "fp16", "e4m3", "e5m2"):
+for _name in ("bf16", "fp16", "e4m3", "e5m2", "b8p4"):
     FMT[_name + "+ieee"] = FMT[_name] | OVF_IEEE
 VARIANT = {"srff": 0, "srf": 1, "src": 2, "rtne": 3, "rta": 4, "rto": 5}
-CODE_DTYPE = {"bf16": np.uint16, "fp16": np.uint16, "e4m3": np.uint8, "e5m2": np.uint8,
-              "bf16+ieee": np.uint16, "fp16+ieee": np.uint16, "e4m3+ieee": np.uint8, "e5m2+ieee": np.uint8}
+CODE_DTYPE = {"bf16": np.uint16, "fp16": np.uint16, "e4m3": np.uint8, "e5m2": np.uint8, "b8p4": np.uint8,
+              "bf16+ieee": np.uint16, "fp16+ieee": np.uint16, "e4m3+ieee": np.uint8, "e5m2+ieee": np.uint8,
+              "b8p4+ieee": np.uint8}
 
 
 class OracleStats(ctypes.Structure):

@@ -45,7 +45,7 @@
 
 typedef unsigned __int128 u128;
 
-enum { FMT_BF16 = 0, FMT_FP16 = 1, FMT_E4M3 = 2, FMT_E5M2 = 3 };
+enum { FMT_BF16 = 0, FMT_FP16 = 1, FMT_E4M3 = 2, FMT_E5M2 = 3, FMT_B8P4 = 4, FMT_COUNT = 5 };
 enum { VAR_SRFF = 0, VAR_SRF = 1, VAR_SRC = 2, VAR_RTNE = 3, VAR_RTA = 4, VAR_RTO = 5 };
 enum { KIND_FINITE = 0, KIND_NAN = 1, KIND_INF = 2, KIND_SAT = 3 };
 
@@ -56,13 +56,17 @@ typedef struct {
     int has_inf;
     uint32_t inf_code;
     uint32_t nan_code;
+    int single_zero;   /* no negative zero: the pattern 1000...0 is the one NaN, and a NaN has no sign */
 } format_t;
 
-static const format_t FORMATS[4] = {
-    /* bf16 */ {16, 8, 127, 0x1.FEp127, 0x7F7Fu, 1, 0x7F80u, 0x7FC0u},
-    /* fp16 */ {16, 11, 15, 65504.0, 0x7BFFu, 1, 0x7C00u, 0x7E00u},
-    /* e4m3 */ {8, 4, 7, 448.0, 0x7Eu, 0, 0u, 0x7Fu},
-    /* e5m2 */ {8, 3, 15, 57344.0, 0x7Bu, 1, 0x7Cu, 0x7Fu},
+static const format_t FORMATS[FMT_COUNT] = {
+    /* bf16 */ {16, 8, 127, 0x1.FEp127, 0x7F7Fu, 1, 0x7F80u, 0x7FC0u, 0},
+    /* fp16 */ {16, 11, 15, 65504.0, 0x7BFFu, 1, 0x7C00u, 0x7E00u, 0},
+    /* e4m3 */ {8, 4, 7, 448.0, 0x7Eu, 0, 0u, 0x7Fu, 0},
+    /* e5m2 */ {8, 3, 15, 57344.0, 0x7Bu, 1, 0x7Cu, 0x7Fu, 0},
+    /* Section IV's target, IEEE WG P3109 Binary8P4: (K, P, B; M) = (8, 4, 8; 224); the all-ones magnitude is
+       the infinity, 0x80 the single NaN, and there is one zero. */
+    /* b8p4 */ {8, 4, 8, 224.0, 0x7Eu, 1, 0x7Fu, 0x80u, 1},
 };
 
 typedef struct {
@@ -135,6 +139,7 @@ float fbsr_oracle_decode(int fmt, uint32_t code)
     uint32_t t = code & ((1u << (f->P - 1)) - 1u);
     uint32_t mag = code & ((1u << (f->K - 1)) - 1u);
     double v;
+    if (f->single_zero && code == f->nan_code) return NAN;
     if (f->has_inf && mag == f->inf_code) v = INFINITY;
     else if ((f->has_inf && mag > f->inf_code) || (!f->has_inf && mag == f->nan_code)) v = NAN;
     else if (e == 0) v = ldexp(0.0 + ldexp((double)t, 1 - f->P), 1 - f->B);
@@ -233,6 +238,7 @@ done:
     if (kind_out) *kind_out = kind;
     if (up_out) *up_out = up;
     if (delta_out) *delta_out = delta;
+    if (f->single_zero && (kind == KIND_NAN || code == 0u)) return code;   /* the NaN and the zero carry no sign */
     return sign | code;
 }
 
@@ -258,7 +264,7 @@ static float arith_result(float y) { return isnan(y) ? NAN : y; }
 
 static int bad_args(int fmt, int variant, int k)
 {
-    return (fmt & ~0x100) < 0 || (fmt & ~0x100) > 3 || variant < 0 || variant > 5 || k < 1 || k > 16;
+    return (fmt & ~0x100) < 0 || (fmt & ~0x100) >= FMT_COUNT || variant < 0 || variant > 5 || k < 1 || k > 16;
 }
 
 /* ------------------------------------------------------------ array forms */

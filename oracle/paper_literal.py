@@ -41,8 +41,12 @@ FORMATS = {
                  max_code=0x7E, inf_code=None, nan_code=0x7F),
     "e5m2": dict(K=8, P=3, B=15, M=Fraction(57344),
                  max_code=0x7B, inf_code=0x7C, nan_code=0x7F),
+    # Section IV's target format, IEEE WG P3109 Binary8P4 = (8, 4, 8; 224): one zero, the pattern 0x80 is
+    # the single NaN (so neither zero nor NaN has a sign), the all-ones magnitude is the infinity.
+    "b8p4": dict(K=8, P=4, B=8, M=Fraction(224),
+                 max_code=0x7E, inf_code=0x7F, nan_code=0x80, single_zero=True),
 }
-FORMAT_IDS = {"bf16": 0, "fp16": 1, "e4m3": 2, "e5m2": 3}
+FORMAT_IDS = {"bf16": 0, "fp16": 1, "e4m3": 2, "e5m2": 3, "b8p4": 4}
 VARIANTS = ("srff", "srf", "src")
 DETERMINISTIC = ("rtne", "rta", "rto")          # Section II-A: ties to even, ties away, ties to odd
 VARIANT_IDS = {"srff": 0, "srf": 1, "src": 2, "rtne": 3, "rta": 4, "rto": 5}
@@ -91,6 +95,8 @@ def decode(fmt, code):
     f = FORMATS[fmt]
     mag = code & ((1 << (f["K"] - 1)) - 1)
     s, e, t = split_code(fmt, code)
+    if f.get("single_zero") and code == f["nan_code"]:
+        return "nan"
     if f["inf_code"] is not None:
         if mag == f["inf_code"]:
             return "-inf" if s else "+inf"
@@ -239,19 +245,22 @@ def round_f32_bits(ybits, fmt, variant, n, N, ieee_overflow=False):
       * NaN  -> the format's quiet NaN, sign kept;
       * +-Inf -> +-Inf, or +-M when the format has no infinity;
       * finite |y| > M -> +-M (saturate); such values are not SR-rounded;
-      * +-0 -> +-0.
+      * +-0 -> +-0;
+      * a format with a single zero (Binary8P4) has no sign on its NaN and none on a zero result, whether
+        the input was -0 or a negative value that rounded down to zero.
     Returns (code, kind, up, delta), kind in {'finite','nan','inf','sat'}.
     """
     f = FORMATS[fmt]
     sign = (ybits >> 31) << (f["K"] - 1)
     mag = ybits & 0x7FFFFFFF
+    single_zero = f.get("single_zero", False)
     if mag > 0x7F800000:
-        return sign | f["nan_code"], "nan", 0, Fraction(0)
+        return (0 if single_zero else sign) | f["nan_code"], "nan", 0, Fraction(0)
     if mag == 0x7F800000:
         code = f["inf_code"] if f["inf_code"] is not None else f["max_code"]
         return sign | code, "inf", 0, Fraction(0)
     if mag == 0:
-        return sign, "finite", 0, Fraction(0)
+        return (0 if single_zero else sign), "finite", 0, Fraction(0)
     xt = f32_bits_to_fraction(mag)
     if xt > f["M"]:
         if ieee_overflow:
@@ -263,6 +272,8 @@ def round_f32_bits(ybits, fmt, variant, n, N, ieee_overflow=False):
                 return sign | (f["inf_code"] if f["inf_code"] is not None else f["nan_code"]), "sat", 0, Fraction(0)
         return sign | f["max_code"], "sat", 0, Fraction(0)
     code, up, delta = round_positive(xt, fmt, variant, n, N)
+    if single_zero and code == 0:
+        return 0, "finite", up, delta
     return sign | code, "finite", up, delta
 
 
