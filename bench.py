@@ -289,7 +289,7 @@ def main():
         x8 = x[: 1 << 27]
         out8 = torch.empty(1 << 27, dtype=torch.uint8, device=dev)
         t8 = {}
-        for fmt in ("e4m3", "e5m2"):
+        for fmt in ("e4m3", "e5m2", "b8p4"):
             for k in (2, 4, 8):
                 a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 fbsr.fbsr_round(x8, fmt, "srf", k, seed=7, scale=2.0 ** -10, out=out8)
@@ -305,7 +305,7 @@ def main():
         codes16 = workloads.lp_sweep(n_local, "bf16", device=dev)
         w8 = torch.empty(n_local, dtype=torch.uint8, device=dev)
         tlp = {}
-        for fmt in ("e4m3", "e5m2"):
+        for fmt in ("e4m3", "e5m2", "b8p4"):
             for variant in VARIANT_LIST:
                 a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 fbsr.fbsr_round_lp(codes16, "bf16", fmt, variant, 3, seed=SEED, out=w8)
@@ -326,6 +326,16 @@ def main():
         b.record(stream)
         torch.cuda.synchronize()
         extras["qat_update_e4m3_bf16_src_k3_GBps"] = round(4.0 * n_local / (a.elapsed_time(b) / 10 * 1e-3) / 1e9, 1)
+        # the same step in Section IV's own format (Binary8P4 weights)
+        fbsr.fbsr_round_lp(codes16, "bf16", "b8p4", "rtne", 1, seed=0, out=w8)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        fbsr.fbsr_qat_update(w8, upd, "b8p4", "bf16", "src", 3, seed=1)
+        a.record(stream)
+        for s_ in range(10):
+            fbsr.fbsr_qat_update(w8, upd, "b8p4", "bf16", "src", 3, seed=2 + s_)
+        b.record(stream)
+        torch.cuda.synchronize()
+        extras["qat_update_b8p4_bf16_src_k3_GBps"] = round(4.0 * n_local / (a.elapsed_time(b) / 10 * 1e-3) / 1e9, 1)
         del codes16, w8, upd
         # fused optimizer step on the 32-block parameter list (22 B/param SGD-momentum, 30 B/param Adam)
         try:

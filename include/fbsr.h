@@ -24,6 +24,8 @@
  *   - The magnitude is rounded and the sign copied.  NaN -> quiet NaN, sign of
  *     the input kept (0x7FC0 bf16, 0x7E00 fp16, 0x7F e4m3 and e5m2).  +-Inf ->
  *     +-Inf, or +-M for e4m3, which has no infinity.  Finite |y| > M -> +-M.
+ *     Binary8P4 has one zero and one NaN: a zero result is 0x00 whatever the sign
+ *     of the input (-0, or a negative value rounded down to zero), NaN -> 0x80.
  *     None of these consume the paper's predicates (Section II leaves values
  *     outside the finite range to deterministic rounding).
  *   - Random draws: Philox4x32-10 with key (seed lo, seed hi).  With
@@ -63,7 +65,9 @@ typedef enum {
     FBSR_BF16 = 0, /* (16,  8, 127; 0x1.FEp127) */
     FBSR_FP16 = 1, /* (16, 11,  15; 65504)      */
     FBSR_E4M3 = 2, /* ( 8,  4,   7; 448)   OCP E4M3: no Inf, S.1111.111 is NaN */
-    FBSR_E5M2 = 3  /* ( 8,  3,  15; 57344) */
+    FBSR_E5M2 = 3, /* ( 8,  3,  15; 57344) */
+    FBSR_B8P4 = 4  /* ( 8,  4,   8; 224)   IEEE WG P3109 Binary8P4, the target of Section IV:
+                      0x7F / 0xFF are +-Inf, 0x80 is the NaN, there is no negative zero */
 } fbsr_fmt;
 
 /* May be or-ed into any `fmt` argument.  Section II says that values beyond the finite range are "rounded
@@ -99,7 +103,7 @@ typedef struct {
 /* ---------------------------------------------------------------------------
  * fbsr_round -- Section II-A/II-B/III-F: dst[i] = FBSR(fl32(src[i] * scale)).
  *   src      device, n binary32 values (read only; must not overlap dst)
- *   dst      device, n codes: uint16 for bf16/fp16, uint8 for e4m3/e5m2
+ *   dst      device, n codes: uint16 for bf16/fp16, uint8 for e4m3/e5m2/b8p4
  *   fmt, variant, k_bits   fbsr_fmt, fbsr_variant, N in 1..16
  *   seed, offset           Philox key and global index of element 0
  *   scale    finite, > 0; the per-tensor factor of a scaled tensor (Section I-A),
@@ -112,7 +116,7 @@ int fbsr_round(const float* src, void* dst, size_t n, int fmt, int variant, int 
  * the source is already a low-precision tensor.  dst[i] = FBSR(fl32(value(src[i]) * scale)), where
  * value() widens the stored code exactly by Eq. (1).
  *   src      device, n codes of src_fmt (FBSR_BF16 or FBSR_FP16, uint16 each); must not overlap dst
- *   dst      device, n codes of dst_fmt (FBSR_E4M3 or FBSR_E5M2, uint8 each)
+ *   dst      device, n codes of dst_fmt (FBSR_E4M3, FBSR_E5M2 or FBSR_B8P4, uint8 each)
  * Other format pairs return FBSR_ERR_UNSUPPORTED.  The fast path needs src and dst 16-byte aligned
  * (8-byte for dst) and `offset` on the tile grid, like fbsr_round.  A NaN source keeps its sign. */
 int fbsr_round_lp(const void* src, int src_fmt, void* dst, size_t n, int dst_fmt, int variant, int k_bits,
@@ -217,7 +221,7 @@ int fbsr_accumulate(void* w_lp, const float* update, size_t n, int fmt, int vari
 
 /* fbsr_qat_update -- Algorithm 1, last line, with the sum formed in the 16-bit format as written there:
  *     w16 = value(w8);  s = RTNE_16(fl32(w16 + u16));  w8 = FBSR(s)          (in place on w8)
- *   w8       device, n codes of w_fmt (FBSR_E4M3 or FBSR_E5M2), read and overwritten
+ *   w8       device, n codes of w_fmt (FBSR_E4M3, FBSR_E5M2 or FBSR_B8P4), read and overwritten
  *   update16 device, n codes of u_fmt (FBSR_BF16 or FBSR_FP16): the update computed in the 16-bit format
  * RTNE_16 rounds to u_fmt with ties to even (saturating); a NaN sum is written as the positive NaN. */
 int fbsr_qat_update(void* w8, const void* update16, size_t n, int w_fmt, int u_fmt, int variant, int k_bits,

@@ -13,11 +13,11 @@ import torch
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_HERE, "libfbsr.so")
 
-FMT = {"bf16": 0, "fp16": 1, "e4m3": 2, "e5m2": 3}
+FMT = {"bf16": 0, "fp16": 1, "e4m3": 2, "e5m2": 3, "b8p4": 4}
 OVF_IEEE = 0x100          # or into a format id, or append "+ieee" to a format name: IEEE overflow instead of saturation
 VARIANT = {"srff": 0, "srf": 1, "src": 2, "rtne": 3, "rta": 4, "rto": 5}
-CODE_DTYPE = {"bf16": torch.uint16, "fp16": torch.uint16, "e4m3": torch.uint8, "e5m2": torch.uint8}
-VIEW_DTYPE = {"bf16": torch.bfloat16, "fp16": torch.float16, "e4m3": torch.float8_e4m3fn,
+CODE_DTYPE = {"bf16": torch.uint16, "fp16": torch.uint16, "e4m3": torch.uint8, "e5m2": torch.uint8, "b8p4": torch.uint8}
+VIEW_DTYPE = {"bf16": torch.bfloat16, "fp16": torch.float16, "e4m3": torch.float8_e4m3fn,    # b8p4: torch has no such dtype
               "e5m2": torch.float8_e5m2}
 
 

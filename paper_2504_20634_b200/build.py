@@ -23,7 +23,7 @@ HEADERS = ["fbsr_device.cuh", "fbsr_kernels.cuh", "fbsr_internal.h", os.path.joi
 
 def _units():
     units = [("fbsr_api.o", "fbsr_api.cu", [])]
-    for fmt in range(4):
+    for fmt in range(5):
         for group in range(3):
             if group == 2 and fmt < 2:
                 continue                      # 16-bit sources are rounded to the 8-bit targets only

@@ -15,10 +15,15 @@ void count_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
 namespace {
 
 typedef int (*dispatch_fn)(const CallArgs&);
-const dispatch_fn kRound[4] = {dispatch_round_0, dispatch_round_1, dispatch_round_2, dispatch_round_3};
-const dispatch_fn kOptim[4] = {dispatch_optim_0, dispatch_optim_1, dispatch_optim_2, dispatch_optim_3};
+const dispatch_fn kRound[5] = {dispatch_round_0, dispatch_round_1, dispatch_round_2, dispatch_round_3, dispatch_round_4};
+const dispatch_fn kOptim[5] = {dispatch_optim_0, dispatch_optim_1, dispatch_optim_2, dispatch_optim_3, dispatch_optim_4};
+inline bool eight_bit(int fmt) { return fmt == FBSR_E4M3 || fmt == FBSR_E5M2 || fmt == FBSR_B8P4; }
+inline int dispatch_lp(int fmt, const CallArgs& a)
+{
+    return fmt == FBSR_E4M3 ? dispatch_lp_2(a) : fmt == FBSR_E5M2 ? dispatch_lp_3(a) : dispatch_lp_4(a);
+}
 
-inline bool bad_enum(int fmt, int variant, int k) { return fmt < 0 || fmt > 3 || variant < 0 || variant > 5 || k < 1 || k > 16; }
+inline bool bad_enum(int fmt, int variant, int k) { return fmt < 0 || fmt > 4 || variant < 0 || variant > 5 || k < 1 || k > 16; }
 // FBSR_OVF_IEEE may be or-ed into a format argument: take it out and report it.
 inline int take_overflow_flag(int& fmt)
 {
@@ -75,9 +80,9 @@ int fbsr_round_lp(const void* src, int src_fmt, void* dst, size_t n, int dst_fmt
                   uint64_t seed, uint64_t offset, float scale, void* cuda_stream)
 {
     const int ovf_ieee = take_overflow_flag(dst_fmt);
-    if (bad_enum(dst_fmt, variant, k_bits) || src_fmt < 0 || src_fmt > 3) return FBSR_ERR_INVALID_ARG;
+    if (bad_enum(dst_fmt, variant, k_bits) || src_fmt < 0 || src_fmt > 4) return FBSR_ERR_INVALID_ARG;
     if (!(scale > 0.0f) || !std::isfinite(scale)) return FBSR_ERR_INVALID_ARG;
-    if ((src_fmt != FBSR_BF16 && src_fmt != FBSR_FP16) || (dst_fmt != FBSR_E4M3 && dst_fmt != FBSR_E5M2))
+    if ((src_fmt != FBSR_BF16 && src_fmt != FBSR_FP16) || !eight_bit(dst_fmt))
         return FBSR_ERR_UNSUPPORTED;
     if (n > 0 && (src == nullptr || dst == nullptr)) return FBSR_ERR_INVALID_ARG;
     if (misaligned(src, 2)) return FBSR_ERR_ALIGNMENT;
@@ -85,7 +90,7 @@ int fbsr_round_lp(const void* src, int src_fmt, void* dst, size_t n, int dst_fmt
     CallArgs a = base_args(OP_ROUND_LP, variant, k_bits, n, seed, offset, dst, cuda_stream);
     a.ovf_ieee = ovf_ieee;
     a.src_lp = src; a.src_fmt = src_fmt; a.scale = scale;
-    return finish(dst_fmt == FBSR_E4M3 ? dispatch_lp_2(a) : dispatch_lp_3(a));
+    return finish(dispatch_lp(dst_fmt, a));
 }
 
 int fbsr_round_mx(const float* src, void* dst, uint8_t* scales, size_t n, int fmt, int variant, int k_bits,
@@ -240,15 +245,15 @@ int fbsr_qat_update(void* w8, const void* update16, size_t n, int w_fmt, int u_f
                     uint64_t seed, uint64_t offset, void* cuda_stream)
 {
     const int ovf_ieee = take_overflow_flag(w_fmt);
-    if (bad_enum(w_fmt, variant, k_bits) || u_fmt < 0 || u_fmt > 3) return FBSR_ERR_INVALID_ARG;
-    if ((w_fmt != FBSR_E4M3 && w_fmt != FBSR_E5M2) || (u_fmt != FBSR_BF16 && u_fmt != FBSR_FP16)) return FBSR_ERR_UNSUPPORTED;
+    if (bad_enum(w_fmt, variant, k_bits) || u_fmt < 0 || u_fmt > 4) return FBSR_ERR_INVALID_ARG;
+    if (!eight_bit(w_fmt) || (u_fmt != FBSR_BF16 && u_fmt != FBSR_FP16)) return FBSR_ERR_UNSUPPORTED;
     if (n > 0 && (!w8 || !update16)) return FBSR_ERR_INVALID_ARG;
     if (misaligned(update16, 2)) return FBSR_ERR_ALIGNMENT;
     if (n == 0) return FBSR_OK;
     CallArgs a = base_args(OP_QAT, variant, k_bits, n, seed, offset, w8, cuda_stream);
     a.ovf_ieee = ovf_ieee;
     a.src_lp = update16; a.src_fmt = u_fmt;
-    return finish(w_fmt == FBSR_E4M3 ? dispatch_lp_2(a) : dispatch_lp_3(a));
+    return finish(dispatch_lp(w_fmt, a));
 }
 
 size_t fbsr_tile_elements(int k_bits)

@@ -18,29 +18,42 @@
 
 namespace fbsr {
 
-enum { BF16 = 0, FP16 = 1, E4M3 = 2, E5M2 = 3 };
+enum { BF16 = 0, FP16 = 1, E4M3 = 2, E5M2 = 3, B8P4 = 4 };
 enum { SRFF = 0, SRF = 1, SRC = 2, RTNE = 3, RTA = 4, RTO = 5 };    // 3..5: Section II-A, no draw
 
+// SINGLE_ZERO: the format has one zero and one NaN (the pattern that would be minus zero); neither has a sign.
 template <int FMT> struct Format;
 template <> struct Format<BF16> {
+    static constexpr bool SINGLE_ZERO = false;
     static constexpr int K = 16, P = 8, EMINB = 1;        // (1 - B) + 127: emin as a binary32 biased exponent
     static constexpr uint32_t MAXBITS = 0x7F7F0000u;       // binary32 pattern of M
     static constexpr uint32_t MAXCODE = 0x7F7Fu, INFCODE = 0x7F80u, NANCODE = 0x7FC0u;
 };
 template <> struct Format<FP16> {
+    static constexpr bool SINGLE_ZERO = false;
     static constexpr int K = 16, P = 11, EMINB = 113;
     static constexpr uint32_t MAXBITS = 0x477FE000u;
     static constexpr uint32_t MAXCODE = 0x7BFFu, INFCODE = 0x7C00u, NANCODE = 0x7E00u;
 };
 template <> struct Format<E4M3> {
+    static constexpr bool SINGLE_ZERO = false;
     static constexpr int K = 8, P = 4, EMINB = 121;
     static constexpr uint32_t MAXBITS = 0x43E00000u;
     static constexpr uint32_t MAXCODE = 0x7Eu, INFCODE = 0x7Eu /* no Inf: saturate */, NANCODE = 0x7Fu;
 };
 template <> struct Format<E5M2> {
+    static constexpr bool SINGLE_ZERO = false;
     static constexpr int K = 8, P = 3, EMINB = 113;
     static constexpr uint32_t MAXBITS = 0x47600000u;
     static constexpr uint32_t MAXCODE = 0x7Bu, INFCODE = 0x7Cu, NANCODE = 0x7Fu;
+};
+// Section IV's target, IEEE WG P3109 Binary8P4 = (8, 4, 8; 224): E4M3's grid at half the scale; the all-ones
+// magnitude is the infinity and 0x80 the NaN.
+template <> struct Format<B8P4> {
+    static constexpr bool SINGLE_ZERO = true;
+    static constexpr int K = 8, P = 4, EMINB = 120;
+    static constexpr uint32_t MAXBITS = 0x43600000u;
+    static constexpr uint32_t MAXCODE = 0x7Eu, INFCODE = 0x7Fu, NANCODE = 0x80u;
 };
 
 // ----------------------------------------------------------------------------
@@ -158,6 +171,9 @@ __device__ __forceinline__ uint32_t round_core(uint32_t ybits, uint32_t n, const
                 if (mag > tie || (mag == tie && (F::MAXCODE & 1u))) enc = FMT == E4M3 ? F::NANCODE : F::INFCODE;
             }
         }
+    }
+    if constexpr (F::SINGLE_ZERO) {
+        if (enc == 0u || enc == F::NANCODE) return enc;       // the zero and the NaN carry no sign
     }
     return enc | sign;
 }
@@ -372,7 +388,10 @@ __device__ __forceinline__ float decode_element(uint32_t code)
         const uint32_t sign = ((code >> (K - 1)) & 1u) << 31;
         const uint32_t mag = code & ((1u << (K - 1)) - 1u);
         const uint32_t e = mag >> (P - 1), t = mag & ((1u << (P - 1)) - 1u);
-        if constexpr (FMT == E4M3) {
+        if constexpr (F::SINGLE_ZERO) {
+            if (code == F::NANCODE) return __uint_as_float(0x7FC00000u);
+            if (mag == F::INFCODE) return __uint_as_float(sign | 0x7F800000u);
+        } else if constexpr (FMT == E4M3) {
             if (mag == F::NANCODE) return __uint_as_float(sign | 0x7FC00000u);
         } else {
             if (mag > F::INFCODE) return __uint_as_float(sign | 0x7FC00000u);

@@ -8,7 +8,7 @@
 #include "fbsr_kernels.cuh"
 
 #ifndef FBSR_FMT
-#error "compile with -DFBSR_FMT=0..3"
+#error "compile with -DFBSR_FMT=0..4"
 #endif
 #ifndef FBSR_GROUP
 #error "compile with -DFBSR_GROUP=0|1|2"
@@ -41,11 +41,12 @@ inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_
 
 [[maybe_unused]] inline bool op_aligned(const MxOp<FMT>& o, size_t h) { return aligned(o.src + h, 32) && h % 32 == 0; }
 [[maybe_unused]] inline MxOp<FMT> op_advance(MxOp<FMT> o, size_t h) { o.src += h; o.scales += h / 32; o.n -= h; return o; }
-template <int UF> inline bool op_aligned(const QatOp<FMT == E4M3 || FMT == E5M2 ? FMT : E4M3, UF>& o, size_t h)
+constexpr int QAT_WF = CODE_BYTES == 1 ? FMT : E4M3;                    // the weight format of the Algorithm-1 step is 8 bits wide
+template <int UF> inline bool op_aligned(const QatOp<QAT_WF, UF>& o, size_t h)
 {
     return aligned(static_cast<const uint16_t*>(o.u16) + h, 32);      // w8 is checked as dst
 }
-template <int UF> inline QatOp<FMT == E4M3 || FMT == E5M2 ? FMT : E4M3, UF> op_advance(QatOp<FMT == E4M3 || FMT == E5M2 ? FMT : E4M3, UF> o, size_t h)
+template <int UF> inline QatOp<QAT_WF, UF> op_advance(QatOp<QAT_WF, UF> o, size_t h)
 {
     o.w8 = static_cast<const uint8_t*>(o.w8) + h; o.u16 = static_cast<const uint16_t*>(o.u16) + h; return o;
 }

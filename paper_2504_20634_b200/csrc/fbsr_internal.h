@@ -44,7 +44,7 @@ constexpr int MAX_SLOW_GRID = 148 * 8;      // CTAs of the general kernel; also 
     int dispatch_round_##fmt(const CallArgs&); \
     int dispatch_optim_##fmt(const CallArgs&);\
     int dispatch_lp_##fmt(const CallArgs&);
-FBSR_DECLARE_DISPATCH(0) FBSR_DECLARE_DISPATCH(1) FBSR_DECLARE_DISPATCH(2) FBSR_DECLARE_DISPATCH(3)
+FBSR_DECLARE_DISPATCH(0) FBSR_DECLARE_DISPATCH(1) FBSR_DECLARE_DISPATCH(2) FBSR_DECLARE_DISPATCH(3) FBSR_DECLARE_DISPATCH(4)
 #undef FBSR_DECLARE_DISPATCH
 
 void count_launch();                         // bumps the counter behind fbsr_launch_count()

@@ -352,12 +352,29 @@ struct AdamOp {
 // Four stored 8-bit codes (one 32-bit word, low byte first) widened exactly to binary32 (Eq. (1)) by way of
 // binary16, which holds every value of both 8-bit formats: E5M2 is the upper byte of a binary16 pattern,
 // E4M3 has a hardware convert for pairs.  NaN codes become NaNs (the sign rule is applied by the caller).
+// Binary8P4 is E4M3's grid at half the scale (exact in binary16), except for the all-ones magnitude (the
+// infinity) and the pattern 0x80 (the NaN), which are patched per byte.
 template <int FMT>
 __device__ __forceinline__ void decode4(uint32_t w, float (&v)[4])
 {
-    static_assert(FMT == E4M3 || FMT == E5M2, "8-bit formats");
+    static_assert(Format<FMT>::K == 8, "8-bit formats");
     uint32_t h01, h23;
-    if constexpr (FMT == E5M2) {
+    if constexpr (FMT == B8P4) {
+        asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h01) : "h"((unsigned short)(w & 0xFFFFu)));
+        asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h23) : "h"((unsigned short)(w >> 16)));
+        const float2 a = __half22float2(*reinterpret_cast<const __half2*>(&h01));
+        const float2 b = __half22float2(*reinterpret_cast<const __half2*>(&h23));
+        const float e[4] = {a.x, a.y, b.x, b.y};
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            const uint32_t code = (w >> (8 * c)) & 0xFFu;
+            float x = __fmul_rn(e[c], 0.5f);
+            if ((code & 0x7Fu) == 0x7Fu) x = __uint_as_float(((code & 0x80u) << 24) | 0x7F800000u);
+            if (code == 0x80u) x = __uint_as_float(0x7FC00000u);
+            v[c] = x;
+        }
+        return;
+    } else if constexpr (FMT == E5M2) {
         h01 = __byte_perm(w, 0u, 0x1404);                  // bytes [0, b0, 0, b1]
         h23 = __byte_perm(w, 0u, 0x3424);                  // bytes [0, b2, 0, b3]
     } else {
@@ -417,7 +434,7 @@ struct AccumOp {
 // Algorithm 1, last line: w16 = value(w8); s = RTNE_16(fl32(w16 + u16)); the caller of finish() rounds s to 8 bits.
 template <int WF, int UF>
 struct QatOp {
-    static_assert((WF == E4M3 || WF == E5M2) && (UF == BF16 || UF == FP16), "8-bit weights, 16-bit updates");
+    static_assert(Format<WF>::K == 8 && (UF == BF16 || UF == FP16), "8-bit weights, 16-bit updates");
     // two octets per lane: 16 weight codes (128 bits) and 16 update codes (256 bits) in, 16 weight codes out
     static constexpr int BATCH = ROW_BATCH >= 2 ? ROW_BATCH / 2 : 1, MIN_CTAS = FBSR_MIN_CTAS_ROUND, OCTETS = 2;
     const void* w8; const void* u16;
@@ -487,7 +504,12 @@ __device__ __forceinline__ void pack_row_fast(const uint32_t (&t)[8], const floa
             const uint32_t c23 = __byte_perm(t[4 * j + 2], t[4 * j + 3], 0x7373);
             const uint32_t s01 = __byte_perm(__float_as_uint(y[4 * j]), __float_as_uint(y[4 * j + 1]), 0x7373);
             const uint32_t s23 = __byte_perm(__float_as_uint(y[4 * j + 2]), __float_as_uint(y[4 * j + 3]), 0x7373);
-            out[j] = __byte_perm(c01, c23, 0x5410) | (__byte_perm(s01, s23, 0x5410) & 0x80808080u);
+            const uint32_t codes = __byte_perm(c01, c23, 0x5410);
+            uint32_t signs = __byte_perm(s01, s23, 0x5410) & 0x80808080u;
+            // one zero only: a zero magnitude takes no sign (bytes are at most 0x7F, so the add carries into
+            // bit 7 of exactly the non-zero ones)
+            if constexpr (Format<FMT>::SINGLE_ZERO) signs &= codes + 0x7F7F7F7Fu;
+            out[j] = codes | signs;
         }
     }
 }

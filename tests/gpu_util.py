@@ -48,7 +48,7 @@ def mixed_inputs(n, seed, fmt):
     ranges, with every special value sprinkled in."""
     from helpers import random_f32, edge_values_f32
     rng = np.random.default_rng(seed)
-    lo, hi = {"bf16": (-126, 127), "fp16": (-30, 17), "e4m3": (-14, 10), "e5m2": (-22, 17)}[fmt]
+    lo, hi = {"bf16": (-126, 127), "fp16": (-30, 17), "e4m3": (-14, 10), "e5m2": (-22, 17), "b8p4": (-15, 9)}[fmt]
     pats = random_f32(rng, n, lo, hi)
     edges = edge_values_f32()
     if n >= 4 * edges.size:

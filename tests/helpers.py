@@ -6,7 +6,8 @@ import numpy as np
 import torch
 
 GOLDEN = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden")
-FMTS = ("bf16", "fp16", "e4m3", "e5m2")
+FMTS = ("bf16", "fp16", "e4m3", "e5m2")       # the formats torch has a dtype for
+ALL_FMTS = FMTS + ("b8p4",)                    # plus Section IV's Binary8P4
 VARIANTS = ("srff", "srf", "src")
 TORCH_DTYPE = {"bf16": torch.bfloat16, "fp16": torch.float16,
                "e4m3": torch.float8_e4m3fn, "e5m2": torch.float8_e5m2}

@@ -5,7 +5,7 @@ import torch
 
 pytestmark = pytest.mark.gpu
 
-from helpers import FMTS, VARIANTS  # noqa: E402
+from helpers import ALL_FMTS as FMTS, VARIANTS  # noqa: E402
 
 
 def setup_module(module):

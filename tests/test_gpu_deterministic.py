@@ -49,7 +49,7 @@ def test_deterministic_modes_everywhere(fmt):
     assert torch.equal(got.view(as_int)[ok], ref[ok])
 
 
-@pytest.mark.parametrize("w_fmt", ["e4m3", "e5m2"])
+@pytest.mark.parametrize("w_fmt", ["e4m3", "e5m2", "b8p4"])
 @pytest.mark.parametrize("u_fmt", ["bf16", "fp16"])
 def test_qat_update(w_fmt, u_fmt):
     rng = np.random.default_rng(95)

@@ -17,7 +17,7 @@ def setup_module(module):
 
 
 @pytest.mark.parametrize("src_fmt", ["bf16", "fp16"])
-@pytest.mark.parametrize("dst_fmt", ["e4m3", "e5m2"])
+@pytest.mark.parametrize("dst_fmt", ["e4m3", "e5m2", "b8p4"])
 def test_every_source_code_every_k(src_fmt, dst_fmt):
     """All 65536 source codes (NaN, Inf, subnormals, saturating values included), shuffled and tiled so that
     several tiles and a ragged tail are covered, every k and variant."""

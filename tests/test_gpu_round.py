@@ -6,7 +6,7 @@ import torch
 
 pytestmark = pytest.mark.gpu
 
-from helpers import FMTS, VARIANTS  # noqa: E402
+from helpers import ALL_FMTS as FMTS, VARIANTS  # noqa: E402
 
 ALL_K = list(range(1, 17))
 
@@ -53,7 +53,7 @@ def test_whole_binary32_exponent_range_and_extreme_scales(fmt):
                 gu.assert_codes_equal(got, expect, "%s %s k=%d scale=%g" % (fmt, variant, k, scale))
 
 
-@pytest.mark.parametrize("fmt", ["bf16", "e4m3"])
+@pytest.mark.parametrize("fmt", ["bf16", "e4m3", "b8p4"])
 def test_small_and_ragged_sizes(fmt):
     for k in (1, 2, 3, 6, 8, 13, 16):
         E = 4 * (32 // k)

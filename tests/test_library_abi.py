@@ -59,6 +59,8 @@ def test_argument_validation_needs_no_device(lib):
     assert lib.fbsr_round(None, None, 8, 0, 0, 4, 0, 0, 1.0, None) == 1        # null pointers with n > 0
     assert lib.fbsr_round(2, 4, 8, 0, 0, 4, 0, 0, 1.0, None) == 3              # src not 4-byte aligned
     assert lib.fbsr_round(None, None, 0, 0, 0, 4, 0, 0, 1.0, None) == 0        # empty call is a no-op
+    assert lib.fbsr_round(None, None, 0, 4, 0, 4, 0, 0, 1.0, None) == 0        # format 4 = Binary8P4
+    assert lib.fbsr_round(None, None, 0, 5, 0, 4, 0, 0, 1.0, None) == 1
 
 
 def test_binding_has_no_fallback():
