@@ -25,6 +25,18 @@ CODE_DTYPE = {"bf16": np.uint16, "fp16": np.uint16, "e4m3": np.uint8, "e5m2": np
               "b8p4+ieee": np.uint8}
 
 
+class OracleDesc(ctypes.Structure):
+    """A format (K, P, B; M) given at run time; see the comment above oracle_desc_t in fbsr_oracle.c."""
+    _fields_ = [("K", ctypes.c_int32), ("P", ctypes.c_int32), ("B", ctypes.c_int32), ("max_code", ctypes.c_uint32),
+                ("has_inf", ctypes.c_int32), ("inf_code", ctypes.c_uint32), ("nan_code", ctypes.c_uint32),
+                ("single_zero", ctypes.c_int32)]
+
+
+def make_desc(K, P, B, max_code, inf_code=None, nan_code=None, single_zero=False):
+    return OracleDesc(K, P, B, max_code, 0 if inf_code is None else 1, 0 if inf_code is None else inf_code,
+                      nan_code, 1 if single_zero else 0)
+
+
 class OracleStats(ctypes.Structure):
     _fields_ = [("n_finite", ctypes.c_uint64), ("n_up", ctypes.c_uint64),
                 ("n_nan", ctypes.c_uint64), ("n_inf", ctypes.c_uint64),
@@ -83,6 +95,16 @@ def lib():
         L.fbsr_oracle_accumulate.argtypes = [vp, vp, sz, i, i, i, u64, u64]
         L.fbsr_oracle_qat_update.argtypes = [vp, vp, sz, i, i, i, i, u64, u64]
         L.fbsr_oracle_qat_update.restype = ctypes.c_int
+        dp = ctypes.POINTER(OracleDesc)
+        L.fbsr_oracle_desc_valid.argtypes = [dp]
+        L.fbsr_oracle_desc_valid.restype = ctypes.c_int
+        L.fbsr_oracle_decode_desc.argtypes = [dp, ctypes.c_uint32]
+        L.fbsr_oracle_decode_desc.restype = ctypes.c_float
+        L.fbsr_oracle_round_one_desc.argtypes = [ctypes.c_float, dp, i, i, i, ctypes.c_uint32, ctypes.POINTER(ctypes.c_int),
+                                                 ctypes.POINTER(ctypes.c_int), ctypes.POINTER(ctypes.c_double)]
+        L.fbsr_oracle_round_one_desc.restype = ctypes.c_uint32
+        L.fbsr_oracle_round_desc.argtypes = [vp, vp, sz, dp, i, i, i, u64, u64, f]
+        L.fbsr_oracle_round_desc.restype = ctypes.c_int
         for name in ("round", "round_bits", "round_stats", "sgd_update", "adam_update", "accumulate"):
             getattr(L, "fbsr_oracle_" + name).restype = ctypes.c_int
         _lib = L
@@ -248,3 +270,26 @@ def fbsr_round_mx(src, fmt, variant, k, seed, offset=0):
     _check(lib().fbsr_oracle_round_mx(_ptr(src), _ptr(dst), _ptr(scales), src.size, FMT[fmt], VARIANT[variant], k,
                                       seed, offset))
     return dst, scales
+
+
+def desc_valid(desc):
+    return bool(lib().fbsr_oracle_desc_valid(ctypes.byref(desc)))
+
+
+def decode_desc(desc, code):
+    return float(lib().fbsr_oracle_decode_desc(ctypes.byref(desc), int(code)))
+
+
+def round_one_desc(y, desc, variant, k, n, ieee_overflow=False):
+    kind, up, delta = ctypes.c_int(), ctypes.c_int(), ctypes.c_double()
+    code = lib().fbsr_oracle_round_one_desc(np.float32(y), ctypes.byref(desc), int(ieee_overflow), VARIANT[variant], k, n,
+                                            ctypes.byref(kind), ctypes.byref(up), ctypes.byref(delta))
+    return int(code), kind.value, up.value, delta.value
+
+
+def fbsr_round_desc(src, desc, variant, k, seed, offset=0, scale=1.0, ieee_overflow=False):
+    src = _f32(src)
+    dst = np.empty(src.size, dtype=np.uint16 if desc.K == 16 else np.uint8)
+    _check(lib().fbsr_oracle_round_desc(_ptr(src), _ptr(dst), src.size, ctypes.byref(desc), int(ieee_overflow),
+                                        VARIANT[variant], k, seed, offset, scale))
+    return dst

@@ -131,9 +131,8 @@ static uint32_t field_of_words(const uint32_t* words, size_t i, int k)
 }
 
 /* ------------------------------------------------------------- Eq. (1) */
-float fbsr_oracle_decode(int fmt, uint32_t code)
+static float decode_f(const format_t* f, uint32_t code)
 {
-    const format_t* f = &FORMATS[fmt & 0xFF];
     uint32_t s = (code >> (f->K - 1)) & 1u;
     uint32_t e = (code >> (f->P - 1)) & ((1u << (f->K - f->P)) - 1u);
     uint32_t t = code & ((1u << (f->P - 1)) - 1u);
@@ -148,16 +147,12 @@ float fbsr_oracle_decode(int fmt, uint32_t code)
     return s ? -r : r;
 }
 
+float fbsr_oracle_decode(int fmt, uint32_t code) { return decode_f(&FORMATS[fmt & 0xFF], code); }
+
 /* ------------------------------------------------ one element, Eq. (2)-(8) */
-uint32_t fbsr_oracle_round_one(float y, int fmt, int variant, int N, uint32_t n,
-                               int* kind_out, int* up_out, double* delta_out)
+static uint32_t round_one_f(float y, const format_t* f, int ieee_overflow, int variant, int N, uint32_t n,
+                            int* kind_out, int* up_out, double* delta_out)
 {
-    /* bit 8 of fmt selects the paper-literal treatment of finite values beyond M (Section II: "rounded
-       deterministically as in IEEE-754 round to nearest"): below M + ulp(M)/2 they give M, from there on
-       the infinity (the NaN code where the format has no infinity).  Without it they saturate to M. */
-    const int ieee_overflow = (fmt >> 8) & 1;
-    fmt &= 0xFF;
-    const format_t* f = &FORMATS[fmt];
     const int P = f->P, B = f->B;
     uint32_t yb = bits_of(y);
     uint32_t sign = (yb >> 31) << (f->K - 1);
@@ -240,6 +235,15 @@ done:
     if (delta_out) *delta_out = delta;
     if (f->single_zero && (kind == KIND_NAN || code == 0u)) return code;   /* the NaN and the zero carry no sign */
     return sign | code;
+}
+
+uint32_t fbsr_oracle_round_one(float y, int fmt, int variant, int N, uint32_t n,
+                               int* kind_out, int* up_out, double* delta_out)
+{
+    /* bit 8 of fmt selects the paper-literal treatment of finite values beyond M (Section II: "rounded
+       deterministically as in IEEE-754 round to nearest"): below M + ulp(M)/2 they give M, from there on
+       the infinity (the NaN code where the format has no infinity).  Without it they saturate to M. */
+    return round_one_f(y, &FORMATS[fmt & 0xFF], (fmt >> 8) & 1, variant, N, n, kind_out, up_out, delta_out);
 }
 
 static void store_code(void* dst, size_t i, int fmt, uint32_t code)
@@ -470,6 +474,69 @@ int fbsr_oracle_accumulate(void* w_lp, const float* update, size_t n, int fmt, i
         float y = arith_result(wv + update[i]);
         uint32_t nr = fbsr_oracle_draw(seed, offset + i, k, 0u);
         store_code(w_lp, i, fmt, fbsr_oracle_round_one(y, fmt, variant, k, nr, 0, 0, 0));
+    }
+    return 0;
+}
+
+/* ------------------------------------------------------------------ formats given at run time
+ * Section II describes a format by (K, P, B; M).  The descriptor carries K, P, B, the code of M, and how the
+ * codes above it are used: has_inf / inf_code (magnitude code of the infinity), nan_code (magnitude code written
+ * for NaN, or the full pattern 1000...0 when single_zero is set), single_zero (one zero, one unsigned NaN).
+ * Accepted: K in {8, 16}; 2 <= P <= min(K - 1, 13); 1 <= B <= 127; exponent of M at most 127. */
+typedef struct {
+    int32_t K, P, B;
+    uint32_t max_code;
+    int32_t has_inf;
+    uint32_t inf_code, nan_code;
+    int32_t single_zero;
+} oracle_desc_t;
+
+static int desc_to_format(const oracle_desc_t* d, format_t* f)
+{
+    if (!d || (d->K != 8 && d->K != 16)) return 1;
+    if (d->P < 2 || d->P > d->K - 1 || d->P > 13) return 1;
+    if (d->B < 1 || d->B > 127) return 1;
+    const uint32_t mag_mask = (1u << (d->K - 1)) - 1u;
+    if (d->max_code == 0u || d->max_code > mag_mask) return 1;
+    if ((int)(d->max_code >> (d->P - 1)) - d->B > 127) return 1;
+    if (d->has_inf && (d->inf_code <= d->max_code || d->inf_code > mag_mask)) return 1;
+    if (d->single_zero) { if (d->nan_code != (1u << (d->K - 1))) return 1; }
+    else if (d->nan_code <= d->max_code || d->nan_code > mag_mask || (d->has_inf && d->nan_code == d->inf_code)) return 1;
+    f->K = d->K; f->P = d->P; f->B = d->B; f->max_code = d->max_code; f->has_inf = d->has_inf;
+    f->inf_code = d->inf_code; f->nan_code = d->nan_code; f->single_zero = d->single_zero;
+    f->M = 0.0;
+    /* M is the value of max_code; decode_f only treats inf_code / nan_code specially, and those lie above it */
+    f->M = (double)decode_f(f, d->max_code);
+    return 0;
+}
+
+int fbsr_oracle_desc_valid(const oracle_desc_t* d) { format_t f; return desc_to_format(d, &f) == 0; }
+
+float fbsr_oracle_decode_desc(const oracle_desc_t* d, uint32_t code)
+{
+    format_t f;
+    if (desc_to_format(d, &f)) return NAN;
+    return decode_f(&f, code);
+}
+
+uint32_t fbsr_oracle_round_one_desc(float y, const oracle_desc_t* d, int ieee_overflow, int variant, int N, uint32_t n,
+                                    int* kind_out, int* up_out, double* delta_out)
+{
+    format_t f;
+    if (desc_to_format(d, &f)) return 0xFFFFFFFFu;
+    return round_one_f(y, &f, ieee_overflow, variant, N, n, kind_out, up_out, delta_out);
+}
+
+int fbsr_oracle_round_desc(const float* src, void* dst, size_t n, const oracle_desc_t* d, int ieee_overflow,
+                           int variant, int k, uint64_t seed, uint64_t offset, float scale)
+{
+    format_t f;
+    if (desc_to_format(d, &f) || variant < 0 || variant > 5 || k < 1 || k > 16) return 1;
+    for (size_t i = 0; i < n; ++i) {
+        float y = scaled(src[i], scale);
+        uint32_t nr = fbsr_oracle_draw(seed, offset + i, k, 0u);
+        uint32_t code = round_one_f(y, &f, ieee_overflow, variant, k, nr, 0, 0, 0);
+        if (f.K == 16) ((uint16_t*)dst)[i] = (uint16_t)code; else ((uint8_t*)dst)[i] = (uint8_t)code;
     }
     return 0;
 }

@@ -52,6 +52,19 @@ DETERMINISTIC = ("rtne", "rta", "rto")          # Section II-A: ties to even, ti
 VARIANT_IDS = {"srff": 0, "srf": 1, "src": 2, "rtne": 3, "rta": 4, "rto": 5}
 
 
+def format_of(fmt):
+    """A format is named (a key of FORMATS) or given outright as a dict with the same fields."""
+    return fmt if isinstance(fmt, dict) else FORMATS[fmt]
+
+
+def make_format(K, P, B, max_code, inf_code=None, nan_code=None, single_zero=False):
+    """A format (K, P, B; M) described at run time, Section II: M is the value of max_code by Eq. (1)."""
+    f = dict(K=K, P=P, B=B, M=None, max_code=max_code, inf_code=inf_code, nan_code=nan_code, single_zero=single_zero)
+    e, t = max_code >> (P - 1), max_code & ((1 << (P - 1)) - 1)
+    f["M"] = value_of(f, 0, e, t)
+    return f
+
+
 def pow2(e):
     """2**e as an exact rational for any integer e."""
     return Fraction(2) ** e
@@ -71,7 +84,7 @@ def floor_log2(x):
 
 def value_of(fmt, s, e, t):
     """F(s, e, t; P, B), Eq. (1): the real value of a finite triple."""
-    f = FORMATS[fmt]
+    f = format_of(fmt)
     P, B = f["P"], f["B"]
     if e == 0:
         mag = (0 + t * pow2(1 - P)) * pow2(1 - B)
@@ -82,7 +95,7 @@ def value_of(fmt, s, e, t):
 
 def split_code(fmt, code):
     """Bit pattern -> (s, e, t)."""
-    f = FORMATS[fmt]
+    f = format_of(fmt)
     K, P = f["K"], f["P"]
     s = (code >> (K - 1)) & 1
     e = (code >> (P - 1)) & ((1 << (K - P)) - 1)
@@ -92,7 +105,7 @@ def split_code(fmt, code):
 
 def decode(fmt, code):
     """Bit pattern -> Fraction, or the strings 'nan' / '+inf' / '-inf'."""
-    f = FORMATS[fmt]
+    f = format_of(fmt)
     mag = code & ((1 << (f["K"] - 1)) - 1)
     s, e, t = split_code(fmt, code)
     if f.get("single_zero") and code == f["nan_code"]:
@@ -205,7 +218,7 @@ def round_positive(xt, fmt, variant, n, N):
     Returns (code_magnitude, up, delta) where up is the predicate's 0/1 value
     and delta the fractional part it was evaluated on.
     """
-    f = FORMATS[fmt]
+    f = format_of(fmt)
     P, B = f["P"], f["B"]
     assert xt > 0 and (variant in DETERMINISTIC or 0 <= n < (1 << N))
     e = max(floor_log2(xt), 1 - B)                     # Eq. (2)
@@ -250,7 +263,7 @@ def round_f32_bits(ybits, fmt, variant, n, N, ieee_overflow=False):
         the input was -0 or a negative value that rounded down to zero.
     Returns (code, kind, up, delta), kind in {'finite','nan','inf','sat'}.
     """
-    f = FORMATS[fmt]
+    f = format_of(fmt)
     sign = (ybits >> 31) << (f["K"] - 1)
     mag = ybits & 0x7FFFFFFF
     single_zero = f.get("single_zero", False)
