@@ -300,6 +300,19 @@ def main():
                 torch.cuda.synchronize()
                 t8["%s/srf/k%d" % (fmt, k)] = round(5.0 * (1 << 27) / (a.elapsed_time(b) / 10 * 1e-3) / 1e9, 1)
         extras["round_fp8_GBps"] = t8
+        # a format described at run time (general kernel): float8_e4m3fnuz = (8, 4, 8; 240), 5 B/element
+        desc = fbsr.format_desc(8, 4, 8, 0x7F, None, 0x80, True)
+        td = {}
+        for k in (3, 8):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            fbsr.fbsr_round_desc(x8, desc, "srf", k, seed=7, scale=2.0 ** -10, out=out8)
+            a.record(stream)
+            for _ in range(5):
+                fbsr.fbsr_round_desc(x8, desc, "srf", k, seed=7, scale=2.0 ** -10, out=out8)
+            b.record(stream)
+            torch.cuda.synchronize()
+            td["(8,4,8;240)/srf/k%d" % k] = round(5.0 * (1 << 27) / (a.elapsed_time(b) / 5 * 1e-3) / 1e9, 1)
+        extras["round_desc_GBps"] = td
         del x8, out8
         # 16-bit sources into 8-bit formats (3 B/element) and the 16-bit-sum weight update (4 B/element)
         codes16 = workloads.lp_sweep(n_local, "bf16", device=dev)

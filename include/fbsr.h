@@ -122,6 +122,39 @@ int fbsr_round(const float* src, void* dst, size_t n, int fmt, int variant, int 
 int fbsr_round_lp(const void* src, int src_fmt, void* dst, size_t n, int dst_fmt, int variant, int k_bits,
                   uint64_t seed, uint64_t offset, float scale, void* cuda_stream);
 
+/* fbsr_round_desc -- fbsr_round for a format (K, P, B; M) given at run time, Section II's parametrisation
+ * ("a binary floating-point format is described by the tuple (K, P, B; M)"); the rounding itself is Section II-A
+ * Eq. (2)-(5) with the predicates of Section II-B and Eq. (8), as in fbsr_round.
+ *   desc     HOST pointer, read before the call returns:
+ *     K          8 or 16: width of a code (dst is uint8 or uint16)
+ *     P          precision including the hidden bit, 2 <= P <= min(K - 1, 13)
+ *     B          exponent bias, 1 <= B <= 127
+ *     max_code   magnitude code of M, the largest finite value (exponent field of M minus B at most 127)
+ *     has_inf / inf_code   whether an infinity exists, and its magnitude code (> max_code)
+ *     nan_code   magnitude code written for NaN (> max_code, != inf_code); with single_zero the pattern
+ *                1 << (K - 1) instead
+ *     single_zero  non-zero: one zero and one unsigned NaN (the pattern that would be minus zero), as in
+ *                Binary8P4; a zero result then has no sign
+ *   ovf_ieee non-zero: finite |y| > M are rounded as IEEE nearest-even does (see FBSR_OVF_IEEE)
+ * Special values follow the conventions at the top of this file (Inf -> the infinity, or +-M without one).
+ * One general kernel serves every descriptor, any alignment and any offset (vector accesses when src is
+ * 16-byte and dst 8 x code-size aligned); it is several times slower than the built-in formats' kernels.
+ * The built-in formats written as descriptors give the built-in results bit for bit.
+ * Returns FBSR_ERR_INVALID_ARG for a descriptor outside the ranges above. */
+typedef struct {
+    int32_t K, P, B;
+    uint32_t max_code;
+    int32_t has_inf;
+    uint32_t inf_code, nan_code;
+    int32_t single_zero;
+} fbsr_format_desc;
+
+int fbsr_round_desc(const float* src, void* dst, size_t n, const fbsr_format_desc* desc, int ovf_ieee,
+                    int variant, int k_bits, uint64_t seed, uint64_t offset, float scale, void* cuda_stream);
+
+/* 1 if fbsr_round_desc accepts the descriptor, else 0.  Host only, no CUDA call. */
+int fbsr_format_desc_valid(const fbsr_format_desc* desc);
+
 /* fbsr_round_mx -- block-scaled tensors (Section I-A: "blocks of low-precision values are accompanied by a
  * scale factor, which may be a power of two").  Blocks are 32 consecutive elements of the call; per block
  *     amax  = largest finite |src| (0 if none)

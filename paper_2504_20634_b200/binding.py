@@ -33,6 +33,19 @@ class FbsrStats(ctypes.Structure):
                 ("sum_e2", ctypes.c_double), ("sum_signed_e", ctypes.c_double), ("sum_abs_e", ctypes.c_double)]
 
 
+class FbsrFormatDesc(ctypes.Structure):
+    """fbsr_format_desc of include/fbsr.h: a format (K, P, B; M) given at run time."""
+    _fields_ = [("K", ctypes.c_int32), ("P", ctypes.c_int32), ("B", ctypes.c_int32), ("max_code", ctypes.c_uint32),
+                ("has_inf", ctypes.c_int32), ("inf_code", ctypes.c_uint32), ("nan_code", ctypes.c_uint32),
+                ("single_zero", ctypes.c_int32)]
+
+
+def format_desc(K, P, B, max_code, inf_code=None, nan_code=0, single_zero=False):
+    """Fill in an FbsrFormatDesc; inf_code=None means that the format has no infinity."""
+    return FbsrFormatDesc(K, P, B, max_code, 0 if inf_code is None else 1, 0 if inf_code is None else inf_code,
+                          nan_code, 1 if single_zero else 0)
+
+
 def _load():
     if not os.path.exists(_LIB_PATH):
         raise ImportError("libfbsr.so is not built: run `python -m paper_2504_20634_b200.build` "
@@ -45,6 +58,10 @@ def _load():
     L.fbsr_round_mx.restype = i
     L.fbsr_round_lp.argtypes = [vp, i, vp, sz, i, i, i, u64, u64, f, vp]
     L.fbsr_round_lp.restype = i
+    L.fbsr_round_desc.argtypes = [vp, vp, sz, ctypes.POINTER(FbsrFormatDesc), i, i, i, u64, u64, f, vp]
+    L.fbsr_round_desc.restype = i
+    L.fbsr_format_desc_valid.argtypes = [ctypes.POINTER(FbsrFormatDesc)]
+    L.fbsr_format_desc_valid.restype = i
     L.fbsr_stats_workspace_bytes.argtypes = []
     L.fbsr_stats_workspace_bytes.restype = sz
     L.fbsr_round_stats.argtypes = [vp, vp, sz, i, i, i, u64, u64, f, sz, vp, vp, vp, vp, sz, vp]
@@ -160,6 +177,22 @@ def fbsr_round_mx(src, fmt, variant, k_bits, seed, offset=0, out=None, scales=No
         _check(_L.fbsr_round_mx(_dev(src, torch.float32, "src"), po, _dev(scales, torch.uint8, "scales"), src.numel(),
                                 _fmt(fmt), _var(variant), k_bits, seed, offset, _stream(src)), "fbsr_round_mx")
     return out, scales
+
+
+def fbsr_round_desc(src, desc, variant, k_bits, seed, offset=0, scale=1.0, ovf_ieee=False, out=None):
+    """fbsr_round for a format described at run time (an FbsrFormatDesc); returns uint8 or uint16 codes."""
+    dt = torch.uint16 if desc.K == 16 else torch.uint8
+    if out is None:
+        out = torch.empty(src.numel(), dtype=dt, device=src.device)
+    with torch.cuda.device(src.device):
+        _check(_L.fbsr_round_desc(_dev(src, torch.float32, "src"), _dev(out, dt, "out"), src.numel(), ctypes.byref(desc),
+                                  1 if ovf_ieee else 0, _var(variant), k_bits, seed, offset, scale, _stream(src)),
+               "fbsr_round_desc")
+    return out
+
+
+def fbsr_format_desc_valid(desc):
+    return bool(_L.fbsr_format_desc_valid(ctypes.byref(desc)))
 
 
 def fbsr_round_lp(src_codes, src_fmt, fmt, variant, k_bits, seed, offset=0, scale=1.0, out=None):

@@ -22,7 +22,7 @@ HEADERS = ["fbsr_device.cuh", "fbsr_kernels.cuh", "fbsr_internal.h", os.path.joi
 
 
 def _units():
-    units = [("fbsr_api.o", "fbsr_api.cu", [])]
+    units = [("fbsr_api.o", "fbsr_api.cu", []), ("fbsr_descriptor.o", "fbsr_descriptor.cu", [])]
     for fmt in range(5):
         for group in range(3):
             if group == 2 and fmt < 2:
@@ -34,7 +34,8 @@ def _units():
 
 def _newest_source():
     paths = [os.path.join(CSRC, h) for h in HEADERS] + [os.path.join(CSRC, "fbsr_api.cu"),
-                                                        os.path.join(CSRC, "fbsr_dispatch.cu"), __file__]
+                                                        os.path.join(CSRC, "fbsr_dispatch.cu"),
+                                                        os.path.join(CSRC, "fbsr_descriptor.cu"), __file__]
     return max(os.path.getmtime(p) for p in paths)
 
 

@@ -24,25 +24,25 @@ enum { SRFF = 0, SRF = 1, SRC = 2, RTNE = 3, RTA = 4, RTO = 5 };    // 3..5: Sec
 // SINGLE_ZERO: the format has one zero and one NaN (the pattern that would be minus zero); neither has a sign.
 template <int FMT> struct Format;
 template <> struct Format<BF16> {
-    static constexpr bool SINGLE_ZERO = false;
+    static constexpr bool SINGLE_ZERO = false, HAS_INF = true;
     static constexpr int K = 16, P = 8, EMINB = 1;        // (1 - B) + 127: emin as a binary32 biased exponent
     static constexpr uint32_t MAXBITS = 0x7F7F0000u;       // binary32 pattern of M
     static constexpr uint32_t MAXCODE = 0x7F7Fu, INFCODE = 0x7F80u, NANCODE = 0x7FC0u;
 };
 template <> struct Format<FP16> {
-    static constexpr bool SINGLE_ZERO = false;
+    static constexpr bool SINGLE_ZERO = false, HAS_INF = true;
     static constexpr int K = 16, P = 11, EMINB = 113;
     static constexpr uint32_t MAXBITS = 0x477FE000u;
     static constexpr uint32_t MAXCODE = 0x7BFFu, INFCODE = 0x7C00u, NANCODE = 0x7E00u;
 };
 template <> struct Format<E4M3> {
-    static constexpr bool SINGLE_ZERO = false;
+    static constexpr bool SINGLE_ZERO = false, HAS_INF = false;
     static constexpr int K = 8, P = 4, EMINB = 121;
     static constexpr uint32_t MAXBITS = 0x43E00000u;
     static constexpr uint32_t MAXCODE = 0x7Eu, INFCODE = 0x7Eu /* no Inf: saturate */, NANCODE = 0x7Fu;
 };
 template <> struct Format<E5M2> {
-    static constexpr bool SINGLE_ZERO = false;
+    static constexpr bool SINGLE_ZERO = false, HAS_INF = true;
     static constexpr int K = 8, P = 3, EMINB = 113;
     static constexpr uint32_t MAXBITS = 0x47600000u;
     static constexpr uint32_t MAXCODE = 0x7Bu, INFCODE = 0x7Cu, NANCODE = 0x7Fu;
@@ -50,10 +50,18 @@ template <> struct Format<E5M2> {
 // Section IV's target, IEEE WG P3109 Binary8P4 = (8, 4, 8; 224): E4M3's grid at half the scale; the all-ones
 // magnitude is the infinity and 0x80 the NaN.
 template <> struct Format<B8P4> {
-    static constexpr bool SINGLE_ZERO = true;
+    static constexpr bool SINGLE_ZERO = true, HAS_INF = true;
     static constexpr int K = 8, P = 4, EMINB = 120;
     static constexpr uint32_t MAXBITS = 0x43600000u;
     static constexpr uint32_t MAXCODE = 0x7Eu, INFCODE = 0x7Fu, NANCODE = 0x80u;
+};
+
+// A format described at run time, Section II's (K, P, B; M): the members of Format<FMT> as data.
+// INFCODE is the code written for an infinite input (the code of M when the format has no infinity).
+struct RtFormat {
+    int K, P, EMINB;
+    uint32_t MAXBITS, MAXCODE, INFCODE, NANCODE;
+    bool SINGLE_ZERO, HAS_INF;
 };
 
 // ----------------------------------------------------------------------------
@@ -95,19 +103,19 @@ struct ElementInfo {
 // One element.  ybits: the (scaled) binary32 pattern; n: the N-bit draw.
 // Returns the K-bit code.  VAR and N are ordinary arguments so that the slow
 // path can pass run-time values; the tiled kernels pass constants and the
-// branches fold away.
+// branches fold away.  The format is an object: Format<FMT> (all members compile-time
+// constants, so everything folds as before) or an RtFormat filled in by the host.
 // ----------------------------------------------------------------------------
-template <int FMT, bool STATS>
-__device__ __forceinline__ uint32_t round_core(uint32_t ybits, uint32_t n, const int VAR, const int N,
-                                               ElementInfo* info, const bool ieee_overflow = false)
+template <class F, bool STATS, bool BF16_SHORTCUT>
+__device__ __forceinline__ uint32_t round_core_fmt(const F f, uint32_t ybits, uint32_t n, const int VAR, const int N,
+                                                   ElementInfo* info, const bool ieee_overflow)
 {
-    using F = Format<FMT>;
-    constexpr int P = F::P;
+    const int P = f.P;
     const uint32_t mag = ybits & 0x7FFFFFFFu;
-    const uint32_t sign = (ybits >> 31) << (F::K - 1);
+    const uint32_t sign = (ybits >> 31) << (f.K - 1);
     uint32_t enc;
 
-    if constexpr (FMT == BF16 && !STATS) {
+    if constexpr (BF16_SHORTCUT) {
         // bfloat16 shares binary32's exponent range: sh is always 16 and the
         // whole of Eq. (2)-(5) is one addition on the magnitude pattern.
         uint32_t t;
@@ -128,7 +136,7 @@ __device__ __forceinline__ uint32_t round_core(uint32_t ybits, uint32_t n, const
         const uint32_t e32 = mag >> 23;
         const uint32_t m = (mag & 0x7FFFFFu) | (e32 ? 0x800000u : 0u);
         const int eb = max((int)e32, 1);
-        const int te = max(eb, F::EMINB);
+        const int te = max(eb, (int)f.EMINB);
         const int sh = (24 - P) + (te - eb);                 // excess bits, >= 24 - P >= 13
         const uint32_t m6 = m << 6;                          // 6 guard positions keep every shift >= 0
         uint32_t sig;
@@ -148,7 +156,7 @@ __device__ __forceinline__ uint32_t round_core(uint32_t ybits, uint32_t n, const
             const uint32_t pre = (m6 + ((1u << (sa - 1)) - 1u) + ((m6 >> sa) & 1u)) >> sa;
             sig = (pre + n) >> N;
         }
-        enc = ((uint32_t)(te - F::EMINB) << (P - 1)) + sig;
+        enc = ((uint32_t)(te - f.EMINB) << (P - 1)) + sig;
         if constexpr (STATS) {
             const uint32_t fl = m >> min(sh, 31);
             const uint32_t r = sh < 32 ? (m & ((1u << sh) - 1u)) : m;
@@ -158,24 +166,31 @@ __device__ __forceinline__ uint32_t round_core(uint32_t ybits, uint32_t n, const
         }
     }
     if constexpr (STATS) info->kind = 0;
-    if (mag > F::MAXBITS) {
-        if (mag > 0x7F800000u) { enc = F::NANCODE; if constexpr (STATS) info->kind = 1; }
-        else if (mag == 0x7F800000u) { enc = F::INFCODE; if constexpr (STATS) info->kind = 2; }
+    if (mag > f.MAXBITS) {
+        if (mag > 0x7F800000u) { enc = f.NANCODE; if constexpr (STATS) info->kind = 1; }
+        else if (mag == 0x7F800000u) { enc = f.INFCODE; if constexpr (STATS) info->kind = 2; }
         else {
             // finite and beyond M: saturate, or (Section II read literally) round as IEEE nearest-even does:
             // M below M + ulp/2, the infinity above it (the NaN code for E4M3), the tie to the even neighbour
-            enc = F::MAXCODE;
+            enc = f.MAXCODE;
             if constexpr (STATS) info->kind = 3;
             if (ieee_overflow) {
-                const uint32_t tie = F::MAXBITS + (1u << (24 - P - 1));
-                if (mag > tie || (mag == tie && (F::MAXCODE & 1u))) enc = FMT == E4M3 ? F::NANCODE : F::INFCODE;
+                const uint32_t tie = f.MAXBITS + (1u << (24 - P - 1));
+                if (mag > tie || (mag == tie && (f.MAXCODE & 1u))) enc = f.HAS_INF ? f.INFCODE : f.NANCODE;
             }
         }
     }
-    if constexpr (F::SINGLE_ZERO) {
-        if (enc == 0u || enc == F::NANCODE) return enc;       // the zero and the NaN carry no sign
+    if (f.SINGLE_ZERO) {
+        if (enc == 0u || enc == f.NANCODE) return enc;        // the zero and the NaN carry no sign
     }
     return enc | sign;
+}
+
+template <int FMT, bool STATS>
+__device__ __forceinline__ uint32_t round_core(uint32_t ybits, uint32_t n, const int VAR, const int N,
+                                               ElementInfo* info, const bool ieee_overflow = false)
+{
+    return round_core_fmt<Format<FMT>, STATS, FMT == BF16 && !STATS>(Format<FMT>{}, ybits, n, VAR, N, info, ieee_overflow);
 }
 
 // ----------------------------------------------------------------------------

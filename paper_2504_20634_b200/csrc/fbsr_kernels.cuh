@@ -364,14 +364,17 @@ __device__ __forceinline__ void decode4(uint32_t w, float (&v)[4])
         asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h23) : "h"((unsigned short)(w >> 16)));
         const float2 a = __half22float2(*reinterpret_cast<const __half2*>(&h01));
         const float2 b = __half22float2(*reinterpret_cast<const __half2*>(&h23));
-        const float e[4] = {a.x, a.y, b.x, b.y};
+        v[0] = __fmul_rn(a.x, 0.5f); v[1] = __fmul_rn(a.y, 0.5f); v[2] = __fmul_rn(b.x, 0.5f); v[3] = __fmul_rn(b.y, 0.5f);
+        // bit 7 of a byte: its magnitude is all ones (the infinity) / its magnitude is zero and its sign is set (the NaN)
+        const uint32_t mag = w & 0x7F7F7F7Fu;
+        const uint32_t special = ((mag + 0x01010101u) | (~(mag + 0x7F7F7F7Fu) & w)) & 0x80808080u;
+        if (special) {
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
-            const uint32_t code = (w >> (8 * c)) & 0xFFu;
-            float x = __fmul_rn(e[c], 0.5f);
-            if ((code & 0x7Fu) == 0x7Fu) x = __uint_as_float(((code & 0x80u) << 24) | 0x7F800000u);
-            if (code == 0x80u) x = __uint_as_float(0x7FC00000u);
-            v[c] = x;
+            for (int c = 0; c < 4; ++c) {
+                const uint32_t code = (w >> (8 * c)) & 0xFFu;
+                if ((code & 0x7Fu) == 0x7Fu) v[c] = __uint_as_float(((code & 0x80u) << 24) | 0x7F800000u);
+                if (code == 0x80u) v[c] = __uint_as_float(0x7FC00000u);
+            }
         }
         return;
     } else if constexpr (FMT == E5M2) {

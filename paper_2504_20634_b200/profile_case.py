@@ -17,7 +17,7 @@ from paper_2504_20634_b200 import workloads
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--op", default="round", choices=["round", "sgd", "adam", "accumulate", "stats", "bits", "lp", "mx"])
+    ap.add_argument("--op", default="round", choices=["round", "sgd", "adam", "accumulate", "stats", "bits", "lp", "mx", "desc"])
     ap.add_argument("--src-fmt", default="bf16", help="source format for --op lp")
     ap.add_argument("--fmt", default="bf16")
     ap.add_argument("--variant", default="srf")
@@ -35,6 +35,15 @@ def main():
     if args.op == "round":
         bytes_per_elem = 4 + code_bytes
         run = lambda s: fbsr.fbsr_round(x, args.fmt, args.variant, args.k, seed=1234, out=out)
+    elif args.op == "desc":
+        # the same format, handed over as a run-time descriptor (general kernel)
+        desc = fbsr.format_desc(*{"bf16": (16, 8, 127, 0x7F7F, 0x7F80, 0x7FC0, False),
+                                  "fp16": (16, 11, 15, 0x7BFF, 0x7C00, 0x7E00, False),
+                                  "e4m3": (8, 4, 7, 0x7E, None, 0x7F, False),
+                                  "e5m2": (8, 3, 15, 0x7B, 0x7C, 0x7F, False),
+                                  "b8p4": (8, 4, 8, 0x7E, 0x7F, 0x80, True)}[args.fmt])
+        bytes_per_elem = 4 + code_bytes
+        run = lambda s: fbsr.fbsr_round_desc(x, desc, args.variant, args.k, seed=1234, out=out)
     elif args.op == "lp":
         codes = workloads.lp_sweep(n, args.src_fmt, device=dev)
         bytes_per_elem = 2 + code_bytes

@@ -70,3 +70,26 @@ def test_binding_has_no_fallback():
         if name.endswith(".py"):
             assert "import oracle" not in open(os.path.join(ROOT, "paper_2504_20634_b200", name)).read()
             assert "from oracle" not in open(os.path.join(ROOT, "paper_2504_20634_b200", name)).read()
+
+
+def test_format_descriptor_validation(lib):
+    """fbsr_format_desc_valid is host-only: the accepted ranges of the header, checked without a GPU."""
+    import ctypes
+
+    class Desc(ctypes.Structure):
+        _fields_ = [("K", ctypes.c_int32), ("P", ctypes.c_int32), ("B", ctypes.c_int32), ("max_code", ctypes.c_uint32),
+                    ("has_inf", ctypes.c_int32), ("inf_code", ctypes.c_uint32), ("nan_code", ctypes.c_uint32),
+                    ("single_zero", ctypes.c_int32)]
+
+    lib.fbsr_format_desc_valid.argtypes = [ctypes.POINTER(Desc)]
+    ok = [(16, 8, 127, 0x7F7F, 1, 0x7F80, 0x7FC0, 0), (8, 4, 7, 0x7E, 0, 0, 0x7F, 0), (8, 4, 8, 0x7E, 1, 0x7F, 0x80, 1),
+          (8, 3, 16, 0x7F, 0, 0, 0x80, 1), (16, 13, 4, 0x7FFE, 0, 0, 0x8000, 1)]
+    bad = [(12, 4, 7, 0x7E, 0, 0, 0x7F, 0), (8, 1, 7, 0x7E, 0, 0, 0x7F, 0), (8, 8, 7, 0x7E, 0, 0, 0x7F, 0),
+           (16, 14, 7, 0x7E, 0, 0, 0x7FFF, 0), (8, 4, 0, 0x7E, 0, 0, 0x7F, 0), (8, 4, 128, 0x7E, 0, 0, 0x7F, 0),
+           (8, 4, 7, 0, 0, 0, 0x7F, 0), (8, 4, 7, 0x7E, 1, 0x7E, 0x7F, 0), (8, 4, 7, 0x7E, 1, 0x7F, 0x7F, 0),
+           (8, 4, 7, 0x7E, 0, 0, 0x7D, 0), (8, 4, 7, 0x7E, 0, 0, 0x7F, 1), (16, 8, 100, 0x7F7F, 1, 0x7F80, 0x7FC0, 0)]
+    for d in ok:
+        assert lib.fbsr_format_desc_valid(ctypes.byref(Desc(*d))) == 1, d
+    for d in bad:
+        assert lib.fbsr_format_desc_valid(ctypes.byref(Desc(*d))) == 0, d
+    assert lib.fbsr_format_desc_valid(None) == 0
