@@ -95,6 +95,8 @@ def lib():
         L.fbsr_oracle_accumulate.argtypes = [vp, vp, sz, i, i, i, u64, u64]
         L.fbsr_oracle_qat_update.argtypes = [vp, vp, sz, i, i, i, i, u64, u64]
         L.fbsr_oracle_qat_update.restype = ctypes.c_int
+        L.fbsr_oracle_qat_adamw_step.argtypes = [vp, vp, vp, vp, sz, i, i, i, i, u64, u64, f, f, f, f, f, i]
+        L.fbsr_oracle_qat_adamw_step.restype = ctypes.c_int
         dp = ctypes.POINTER(OracleDesc)
         L.fbsr_oracle_desc_valid.argtypes = [dp]
         L.fbsr_oracle_desc_valid.restype = ctypes.c_int
@@ -259,6 +261,14 @@ def qat_update(w8, u16, w_fmt, u_fmt, variant, k, seed, offset=0):
     u16 = np.ascontiguousarray(u16, dtype=np.uint16)
     _check(lib().fbsr_oracle_qat_update(_ptr(w8), _ptr(u16), w8.size, FMT[w_fmt], FMT[u_fmt], VARIANT[variant], k,
                                         seed, offset))
+    return w8
+
+
+def qat_adamw_step(w8, g16, m, v, w_fmt, g_fmt, variant, k, seed, offset, lr, beta1, beta2, eps, weight_decay, step):
+    """In place on w8 (uint8 codes), m and v (float32)."""
+    assert w8.dtype == np.uint8 and g16.dtype == np.uint16 and m.dtype == np.float32 and v.dtype == np.float32
+    _check(lib().fbsr_oracle_qat_adamw_step(_ptr(w8), _ptr(g16), _ptr(m), _ptr(v), w8.size, FMT[w_fmt], FMT[g_fmt],
+                                            VARIANT[variant], k, seed, offset, lr, beta1, beta2, eps, weight_decay, step))
     return w8
 
 

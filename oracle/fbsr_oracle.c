@@ -463,6 +463,48 @@ int fbsr_oracle_qat_update(void* w8, const void* u16, size_t n, int w_fmt, int u
     return 0;
 }
 
+/* Algorithm 1, one whole iteration per parameter, from the gradient on:
+ *   w16 = value(w8)  (exact);  g = value(g16);
+ *   "AdamW update in F16": moments in binary32, every operation rounded once, the result rounded to F16:
+ *     m' = fma(b1, m, a1 g);  v' = fma(b2, v, (a2 g) g);  d = sqrt(v') c2 + eps;
+ *     u32 = fma(-c1, m'/d, -(lr wd) w16);   u16 = RTNE_F16(u32)          (c1, c2, a1, a2 as for Adam)
+ *   w8' = FBSR(RTNE_F16(fl32(w16 + u16)))                                 (the step above)
+ * The paper gives no arithmetic for the update; this operation list is the library's definition. */
+int fbsr_oracle_qat_adamw_step(void* w8, const void* g16, float* m, float* v, size_t n, int w_fmt, int g_fmt,
+                               int variant, int k, uint64_t seed, uint64_t offset, float lr, float beta1,
+                               float beta2, float eps, float weight_decay, int step)
+{
+    if (bad_args(w_fmt, variant, k) || g_fmt < 0 || g_fmt > 1 || (w_fmt & 0xFF) < 2 || step < 1) return 1;
+    float c[4];
+    fbsr_oracle_adam_coefficients(lr, beta1, beta2, step, c);
+    const float c1 = c[0], c2 = c[1], a1 = c[2], a2 = c[3];
+    const float lrwd = lr * weight_decay;
+    for (size_t i = 0; i < n; ++i) {
+        float wv = fbsr_oracle_decode(w_fmt, load_code(w8, i, w_fmt));
+        float gv = fbsr_oracle_decode(g_fmt, load_code(g16, i, g_fmt));
+        float a1g = a1 * gv;
+        float m2 = fmaf(beta1, m[i], a1g);
+        float a2g = a2 * gv;
+        float a2gg = a2g * gv;
+        float v2 = fmaf(beta2, v[i], a2gg);
+        float sq = sqrtf(v2);
+        float sc = sq * c2;
+        float d = sc + eps;
+        float qt = m2 / d;
+        float decay = -lrwd * wv;
+        float u32 = fmaf(-c1, qt, decay);
+        m[i] = m2; v[i] = v2;
+        uint32_t u16 = fbsr_oracle_round_one(arith_result(u32), g_fmt, VAR_RTNE, 1, 0u, 0, 0, 0);
+        float uv = fbsr_oracle_decode(g_fmt, u16);
+        float s32 = arith_result(wv + uv);
+        uint32_t s16 = fbsr_oracle_round_one(s32, g_fmt, VAR_RTNE, 1, 0u, 0, 0, 0);
+        float y = arith_result(fbsr_oracle_decode(g_fmt, s16));
+        uint32_t nr = fbsr_oracle_draw(seed, offset + i, k, 0u);
+        store_code(w8, i, w_fmt, fbsr_oracle_round_one(y, w_fmt, variant, k, nr, 0, 0, 0));
+    }
+    return 0;
+}
+
 /* Low-precision accumulation (last line of Algorithm 1): the stored weight is
  * widened exactly, the update added in binary32, the sum SR-rounded back. */
 int fbsr_oracle_accumulate(void* w_lp, const float* update, size_t n, int fmt, int variant, int k,

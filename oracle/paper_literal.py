@@ -485,6 +485,27 @@ def adam_coefficients(lr_bits, beta1_bits, beta2_bits, step):
     return b(lr / (1.0 - b1t)), b(1.0 / math.sqrt(1.0 - b2t)), b(1.0 - b1), b(1.0 - b2)
 
 
+def qat_adamw_step(w8, g16, m, v, w_fmt, g_fmt, variant, n, N, beta1, beta2, eps, c1, c2, a1, a2, lrwd):
+    """One iteration of Algorithm 1 for one finite parameter, every step exact and rounded once.
+
+    w8, g16: stored codes; m, v and the scalars: binary32 patterns (lrwd = fl32(lr * weight_decay)).
+    Returns (new w8 code, m', v', u16 code).  Same operation list as the C tier:
+    u32 = fma(-c1, m'/d, -(lrwd) w16), u16 = RTNE_F16(u32), s16 = RTNE_F16(fl32(w16 + u16)), w8' = FBSR(s16).
+    """
+    wbits = fraction_to_f32_bits(decode(w_fmt, w8), negative_zero=bool(w8 >> (format_of(w_fmt)["K"] - 1)) and decode(w_fmt, w8) == 0)
+    gbits = fraction_to_f32_bits(decode(g_fmt, g16), negative_zero=bool(g16 >> 15) and decode(g_fmt, g16) == 0)
+    m2 = _fma(beta1, m, _mul(a1, gbits))
+    v2 = _fma(beta2, v, _mul(_mul(a2, gbits), gbits))
+    d = _add(_mul(_sqrt(v2), c2), eps)
+    u32 = _fma(_neg(c1), _div(m2, d), _mul(_neg(lrwd), wbits))
+    u16 = round_f32_bits(u32, g_fmt, "rtne", 0, 1)[0]
+    ubits = fraction_to_f32_bits(decode(g_fmt, u16), negative_zero=bool(u16 >> 15) and decode(g_fmt, u16) == 0)
+    s32 = _add(wbits, ubits)
+    s16 = round_f32_bits(s32, g_fmt, "rtne", 0, 1)[0]
+    sbits = fraction_to_f32_bits(decode(g_fmt, s16), negative_zero=bool(s16 >> 15) and decode(g_fmt, s16) == 0)
+    return round_f32_bits(sbits, w_fmt, variant, n, N)[0], m2, v2, u16
+
+
 def adam_step(w, g, m, v, beta1, beta2, eps, c1, c2, a1, a2):
     """m' = fma(b1, m, a1*g); v' = fma(b2, v, (a2*g)*g);
     d = sqrt(v')*c2 + eps;  w' = fma(-c1, m'/d, w)."""
