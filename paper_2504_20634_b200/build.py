@@ -39,8 +39,13 @@ def _newest_source():
     return max(os.path.getmtime(p) for p in paths)
 
 
-def _compile(unit, verbose):
+def _compile(unit, verbose, force=False):
     obj, src, defs = unit
+    # an object newer than the headers, its own source and this file is kept
+    deps = [os.path.join(CSRC, h) for h in HEADERS] + [os.path.join(CSRC, src), __file__]
+    out = os.path.join(OBJ, obj)
+    if not force and not verbose and os.path.exists(out) and os.path.getmtime(out) >= max(os.path.getmtime(d) for d in deps):
+        return obj, ""
     cmd = [NVCC, *FLAGS, *(["-Xptxas", "-v"] if verbose else []), *defs, "-c", os.path.join(CSRC, src),
            "-o", os.path.join(OBJ, obj)]
     res = subprocess.run(cmd, capture_output=True, text=True)
@@ -56,7 +61,7 @@ def build(force=False, verbose=False):
     os.makedirs(OBJ, exist_ok=True)
     units = _units()
     with concurrent.futures.ThreadPoolExecutor(max_workers=min(len(units), os.cpu_count() or 4)) as pool:
-        for obj, log in pool.map(lambda u: _compile(u, verbose), units):
+        for obj, log in pool.map(lambda u: _compile(u, verbose, force), units):
             if verbose:
                 with open(os.path.join(OBJ, obj + ".ptxas.txt"), "w") as fh:
                     fh.write(log)

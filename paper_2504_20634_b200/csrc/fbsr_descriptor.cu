@@ -1,7 +1,13 @@
 // fbsr_round_desc: rounding to a format (K, P, B; M) that is described at run time (Section II).
-// One kernel for every such format: the element-wise integer rounder with the format's constants as
-// kernel arguments.  A thread takes 8 consecutive elements (vector accesses when the pointers allow),
-// and computes the one or two generator calls that cover them from their global indices.
+// One kernel for every such format, with the format's constants as kernel arguments.  A thread takes 8
+// consecutive elements (vector accesses when the pointers allow) and computes the one or two generator
+// calls that cover them from their global indices.
+// Rounding: as in the tiled kernels, |y| is first multiplied by 2^(1 - EMINB), toward zero, so that the
+// target's exponent range starts where binary32's does; then Eq. (2)-(5) are one addition on the pattern
+// with sh0 = 24 - P excess bits: code = (pattern + (n << (sh0 - N))) >> sh0.  This needs N <= sh0 excess
+// bits (one more for SRF's half step, two more for SRC's pre-round).  Finite values beyond M saturate by a
+// min on the pattern.  Wider draws, Inf, NaN and, with the IEEE overflow option, every value beyond M go
+// through the element-wise integer rounder.
 #include <cmath>
 #include <cstring>
 
@@ -15,12 +21,23 @@ namespace {
 constexpr int DESC_THREADS = 256;
 
 __global__ void __launch_bounds__(DESC_THREADS)
-descriptor_kernel(const float* __restrict__ src, void* __restrict__ dst, const uint64_t n, const uint64_t offset,
-                  const float scale, const RtFormat f, const int variant, const int k, const uint32_t k0,
+descriptor_kernel(const float* __restrict__ src, void* __restrict__ dst, const uint64_t n, const uint64_t call_base,
+                  const uint32_t first_field, const bool short_call, const float scale, const RtFormat f, const int variant, const int k, const uint32_t k0,
                   const uint32_t k1, const bool ieee_overflow, const bool vectors)
 {
     const uint32_t dpw = 32u / (uint32_t)k, E = 4u * dpw, mask = (1u << k) - 1u;      // E >= 8
     const bool draws = variant < RTNE;
+    // the one-addition form and its constants
+    const int sh0 = 24 - f.P;                                                           // >= 11
+    const int needed = variant == SRF ? k + 1 : variant == SRC ? k + 2 : k;
+    const bool one_addition = !draws || needed <= sh0;
+    const int pos = draws ? sh0 - k : sh0;                   // where the draw (or the half step) is added
+    const uint32_t half = one_addition && pos > 0 ? 1u << (pos - 1) : 0u;
+    const uint32_t below_half = half ? half - 1u : 0u;
+    const bool sticky = variant == SRC || variant == RTNE || variant == RTO;
+    const uint32_t flip = variant == RTO ? 1u : 0u;
+    const float rescale = __uint_as_float((uint32_t)(128 - f.EMINB) << 23);            // 2^(1 - EMINB)
+    const uint32_t max_pattern = f.MAXCODE << sh0;                                      // rescaled pattern of M
     const uint64_t n_octets = (n + 7) / 8;
     for (uint64_t o = (uint64_t)blockIdx.x * DESC_THREADS + threadIdx.x; o < n_octets;
          o += (uint64_t)gridDim.x * DESC_THREADS) {
@@ -36,24 +53,48 @@ descriptor_kernel(const float* __restrict__ src, void* __restrict__ dst, const u
 #pragma unroll
             for (int c = 0; c < 8; ++c) x[c] = c < cnt ? src[i0 + c] : 0.0f;
         }
-        const uint64_t g0 = offset + i0, call = g0 / E;
-        const uint32_t j0 = (uint32_t)(g0 - call * E);
+        // global index of element i0 = call_base * E + first_field + i0; a 32-bit division when the call is short
+        const uint64_t rel = (uint64_t)first_field + i0;
+        const uint64_t q = short_call ? (uint64_t)((uint32_t)rel / E) : rel / E;
+        const uint64_t call = call_base + q;
+        const uint32_t j0 = (uint32_t)(rel - q * E);
         uint4 a = make_uint4(0u, 0u, 0u, 0u), b = a;
         if (draws) {
             a = philox_block(call, k0, k1);
             b = (j0 + 7 >= E) ? philox_block(call + 1, k0, k1) : a;
         }
+        // word and field of the first element; the following ones are reached by stepping, without divisions
+        uint32_t ws = j0 / dpw, shift = (j0 - ws * dpw) * (uint32_t)k;
+        const uint32_t shift_end = dpw * (uint32_t)k;
+        uint4 cur = a;
         uint32_t codes[8];
 #pragma unroll
         for (int c = 0; c < 8; ++c) {
-            uint32_t j = j0 + c;
-            const uint4 w4 = j < E ? a : b;
-            j = j < E ? j : j - E;
-            const uint32_t ws = j / dpw;
-            const uint32_t word = ws == 0 ? w4.x : ws == 1 ? w4.y : ws == 2 ? w4.z : w4.w;
-            const uint32_t nr = (word >> ((j - ws * dpw) * (uint32_t)k)) & mask;
-            codes[c] = round_core_fmt<RtFormat, false, false>(f, scaled_bits(x[c], scale), nr, variant, k, nullptr,
-                                                              ieee_overflow);
+            const uint32_t word = ws == 0 ? cur.x : ws == 1 ? cur.y : ws == 2 ? cur.z : cur.w;
+            const uint32_t nr = (word >> shift) & mask;
+            const uint32_t yb = scaled_bits(x[c], scale);
+            const uint32_t mbits = yb & 0x7FFFFFFFu;
+            if (one_addition && mbits <= (ieee_overflow ? f.MAXBITS : 0x7F7FFFFFu)) {
+                const float mag = __uint_as_float(mbits);
+                uint32_t u = __float_as_uint(__fmul_rz(mag, rescale));
+                if (sticky) u |= (u ^ __float_as_uint(__fmul_ru(mag, rescale))) & 1u;   // what the truncation lost
+                u = min(u, max_pattern);                     // finite values beyond M saturate: nothing added below can carry past M
+                uint32_t sum;
+                if (variant == SRFF) sum = u + (nr << pos);
+                else if (variant == SRF) sum = u + half + (nr << pos);
+                else if (variant == RTA) sum = u + half;
+                else sum = u + below_half + (((u >> pos) & 1u) ^ flip) + (draws ? nr << pos : 0u);
+                const uint32_t code = sum >> sh0;
+                const uint32_t sign = (yb >> 31) << (f.K - 1);
+                codes[c] = (f.SINGLE_ZERO && code == 0u) ? 0u : (code | sign);
+            } else {
+                codes[c] = round_core_fmt<RtFormat, false, false>(f, yb, nr, variant, k, nullptr, ieee_overflow);
+            }
+            shift += (uint32_t)k;
+            if (shift == shift_end) {
+                shift = 0u;
+                if (++ws == 4u) { ws = 0u; cur = b; }
+            }
         }
         if (whole) {
             if (f.K == 16) {
@@ -132,8 +173,11 @@ extern "C" int fbsr_round_desc(const float* src, void* dst, size_t n, const fbsr
     const uint64_t n_octets = ((uint64_t)n + 7) / 8;
     const uint64_t want = (n_octets + DESC_THREADS - 1) / DESC_THREADS;
     const unsigned grid = (unsigned)(want < 0x7FFFFFF0ull ? want : 0x7FFFFFF0ull);
+    const uint32_t E = 4u * (32u / (uint32_t)k_bits);
+    const uint32_t first_field = (uint32_t)(offset % E);
+    const bool short_call = (uint64_t)n + first_field + 8u < 0xFFFFFFFFull;
     descriptor_kernel<<<grid, DESC_THREADS, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
-        src, dst, (uint64_t)n, offset, scale, f, variant, k_bits, (uint32_t)seed, (uint32_t)(seed >> 32),
+        src, dst, (uint64_t)n, offset / E, first_field, short_call, scale, f, variant, k_bits, (uint32_t)seed, (uint32_t)(seed >> 32),
         ovf_ieee != 0, vectors);
     count_launch();
     return cudaGetLastError() == cudaSuccess ? FBSR_OK : FBSR_ERR_CUDA;
