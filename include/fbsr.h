@@ -252,6 +252,21 @@ int fbsr_adam_update(float* master_w, const float* grad, float* m, float* v, voi
 int fbsr_accumulate(void* w_lp, const float* update, size_t n, int fmt, int variant, int k_bits,
                     uint64_t seed, uint64_t offset, void* cuda_stream);
 
+/* fbsr_qat_adamw_step -- Algorithm 1, one whole iteration from the gradient on, fused:
+ *     w16 = value(w8);  g = value(grad16);
+ *     "AdamW update in F16": moments in binary32, each operation rounded once, the result rounded to the 16-bit format
+ *         m' = fma(beta1, m, a1 g);  v' = fma(beta2, v, (a2 g) g);  d = sqrt(v') c2 + eps;
+ *         u32 = fma(-c1, m' / d, -(lr weight_decay) w16);   u16 = RTNE_16(u32)      (c1, c2, a1, a2 as in fbsr_adam_update)
+ *     w8 = FBSR(RTNE_16(fl32(w16 + u16)))                                            (as in fbsr_qat_update; SR applied here)
+ *   w8       device, n codes of w_fmt (FBSR_E4M3, FBSR_E5M2 or FBSR_B8P4), read and overwritten
+ *   grad16   device, n codes of g_fmt (FBSR_BF16 or FBSR_FP16), the "F16" of the algorithm
+ *   m, v     device, n binary32 moments each, read and overwritten
+ * 20 bytes per parameter.  The paper states the shape of the step, not its arithmetic: the operation list is this
+ * library's.  A NaN result is written as the positive NaN code; m and v then hold NaNs of unspecified sign. */
+int fbsr_qat_adamw_step(void* w8, const void* grad16, float* m, float* v, size_t n, int w_fmt, int g_fmt, int variant,
+                        int k_bits, uint64_t seed, uint64_t offset, float lr, float beta1, float beta2, float eps,
+                        float weight_decay, int step, void* cuda_stream);
+
 /* fbsr_qat_update -- Algorithm 1, last line, with the sum formed in the 16-bit format as written there:
  *     w16 = value(w8);  s = RTNE_16(fl32(w16 + u16));  w8 = FBSR(s)          (in place on w8)
  *   w8       device, n codes of w_fmt (FBSR_E4M3, FBSR_E5M2 or FBSR_B8P4), read and overwritten

@@ -11,7 +11,7 @@ import importlib
 _BINDING_NAMES = (
     "FMT", "VARIANT", "CODE_DTYPE", "VIEW_DTYPE", "FbsrError", "fbsr_round", "fbsr_round_bits", "fbsr_round_lp", "fbsr_round_mx",
     "fbsr_round_desc", "fbsr_format_desc_valid", "FbsrFormatDesc", "format_desc",
-    "fbsr_round_stats", "fbsr_round_stats_noalloc", "stats_from_bytes", "fbsr_sgd_update", "fbsr_adam_update", "fbsr_accumulate", "fbsr_qat_update", "fbsr_round_host",
+    "fbsr_round_stats", "fbsr_round_stats_noalloc", "stats_from_bytes", "fbsr_sgd_update", "fbsr_adam_update", "fbsr_accumulate", "fbsr_qat_update", "fbsr_qat_adamw_step", "fbsr_round_host",
     "fbsr_tile_elements", "fbsr_launch_count", "fbsr_stats_workspace_bytes",
     "fbsr_round_host_min_workspace", "fbsr_version", "fbsr_status_string", "library_path",
 )

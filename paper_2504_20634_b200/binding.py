@@ -72,6 +72,8 @@ def _load():
     L.fbsr_accumulate.argtypes = [vp, vp, sz, i, i, i, u64, u64, vp]
     L.fbsr_qat_update.argtypes = [vp, vp, sz, i, i, i, i, u64, u64, vp]
     L.fbsr_qat_update.restype = i
+    L.fbsr_qat_adamw_step.argtypes = [vp, vp, vp, vp, sz, i, i, i, i, u64, u64, f, f, f, f, f, i, vp]
+    L.fbsr_qat_adamw_step.restype = i
     L.fbsr_round_host_min_workspace.argtypes = []
     L.fbsr_round_host_min_workspace.restype = sz
     L.fbsr_round_host.argtypes = [vp, vp, sz, i, i, i, u64, u64, f, vp, sz, vp]
@@ -294,6 +296,17 @@ def fbsr_qat_update(w8, update16, w_fmt, u_fmt, variant, k_bits, seed, offset=0)
         _check(_L.fbsr_qat_update(_dev(w8, torch.uint8, "w8"), _dev(update16, torch.uint16, "update16"), w8.numel(),
                                   _fmt(w_fmt), _fmt(u_fmt), _var(variant), k_bits, seed, offset, _stream(w8)),
                "fbsr_qat_update")
+    return w8
+
+
+def fbsr_qat_adamw_step(w8, grad16, m, v, w_fmt, g_fmt, variant, k_bits, seed, offset, lr, beta1, beta2, eps,
+                        weight_decay, step):
+    """One iteration of Algorithm 1, in place on w8 (uint8 codes), m and v (float32); grad16 holds g_fmt codes."""
+    with torch.cuda.device(w8.device):
+        _check(_L.fbsr_qat_adamw_step(_dev(w8, torch.uint8, "w8"), _dev(grad16, torch.uint16, "grad16"),
+                                      _dev(m, torch.float32, "m"), _dev(v, torch.float32, "v"), w8.numel(), _fmt(w_fmt),
+                                      _fmt(g_fmt), _var(variant), k_bits, seed, offset, lr, beta1, beta2, eps, weight_decay,
+                                      step, _stream(w8)), "fbsr_qat_adamw_step")
     return w8
 
 

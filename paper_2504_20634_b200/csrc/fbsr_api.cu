@@ -256,6 +256,32 @@ int fbsr_qat_update(void* w8, const void* update16, size_t n, int w_fmt, int u_f
     return finish(dispatch_lp(w_fmt, a));
 }
 
+int fbsr_qat_adamw_step(void* w8, const void* grad16, float* m, float* v, size_t n, int w_fmt, int g_fmt, int variant,
+                        int k_bits, uint64_t seed, uint64_t offset, float lr, float beta1, float beta2, float eps,
+                        float weight_decay, int step, void* cuda_stream)
+{
+    const int ovf_ieee = take_overflow_flag(w_fmt);
+    if (bad_enum(w_fmt, variant, k_bits) || g_fmt < 0 || g_fmt > 4 || step < 1) return FBSR_ERR_INVALID_ARG;
+    if (!eight_bit(w_fmt) || (g_fmt != FBSR_BF16 && g_fmt != FBSR_FP16)) return FBSR_ERR_UNSUPPORTED;
+    if (n > 0 && (!w8 || !grad16 || !m || !v)) return FBSR_ERR_INVALID_ARG;
+    if (misaligned(grad16, 2) || misaligned(m, 4) || misaligned(v, 4)) return FBSR_ERR_ALIGNMENT;
+    if (n == 0) return FBSR_OK;
+    double b1t = 1.0, b2t = 1.0;
+    for (int t = 0; t < step; ++t) { b1t *= (double)beta1; b2t *= (double)beta2; }
+    CallArgs a = base_args(OP_QAT_ADAMW, variant, k_bits, n, seed, offset, w8, cuda_stream);
+    a.ovf_ieee = ovf_ieee;
+    a.src_lp = grad16; a.src_fmt = g_fmt; a.m = m; a.v = v;
+    a.beta1 = beta1; a.beta2 = beta2; a.eps = eps;
+    a.neg_c1 = -(float)((double)lr / (1.0 - b1t));
+    a.c2 = (float)(1.0 / std::sqrt(1.0 - b2t));
+    a.a1 = (float)(1.0 - (double)beta1);
+    a.a2 = (float)(1.0 - (double)beta2);
+    const volatile float lrwd = lr * weight_decay;           // one rounded binary32 product
+    a.neg_lrwd = -lrwd;
+    return finish(w_fmt == FBSR_E4M3 ? dispatch_qat_adamw_2(a) : w_fmt == FBSR_E5M2 ? dispatch_qat_adamw_3(a)
+                                                                                   : dispatch_qat_adamw_4(a));
+}
+
 size_t fbsr_tile_elements(int k_bits)
 {
     if (k_bits < 1 || k_bits > 16) return 0;

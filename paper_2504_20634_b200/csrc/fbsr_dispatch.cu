@@ -11,7 +11,7 @@
 #error "compile with -DFBSR_FMT=0..4"
 #endif
 #ifndef FBSR_GROUP
-#error "compile with -DFBSR_GROUP=0|1|2"
+#error "compile with -DFBSR_GROUP=0|1|2|3"
 #endif
 
 namespace fbsr {
@@ -49,6 +49,14 @@ template <int UF> inline bool op_aligned(const QatOp<QAT_WF, UF>& o, size_t h)
 template <int UF> inline QatOp<QAT_WF, UF> op_advance(QatOp<QAT_WF, UF> o, size_t h)
 {
     o.w8 = static_cast<const uint8_t*>(o.w8) + h; o.u16 = static_cast<const uint16_t*>(o.u16) + h; return o;
+}
+template <int UF> inline bool op_aligned(const QatAdamOp<QAT_WF, UF>& o, size_t h)
+{
+    return aligned(static_cast<const uint16_t*>(o.g16) + h, 16) && aligned(o.m + h, 32) && aligned(o.v + h, 32);   // w8 is checked as dst
+}
+template <int UF> inline QatAdamOp<QAT_WF, UF> op_advance(QatAdamOp<QAT_WF, UF> o, size_t h)
+{
+    o.w8 = static_cast<const uint8_t*>(o.w8) + h; o.g16 = static_cast<const uint16_t*>(o.g16) + h; o.m += h; o.v += h; return o;
 }
 template <int SRC> inline bool op_aligned(const LpSrcOp<SRC>& o, size_t h)
 {
@@ -225,6 +233,20 @@ int FBSR_CAT(dispatch_lp_, FBSR_FMT)(const CallArgs& a)
     }
     if (a.src_fmt == BF16) return by_variant_and_k<LpSrcOp<BF16>, false>(LpSrcOp<BF16>{a.src_lp, a.scale}, a);
     if (a.src_fmt == FP16) return by_variant_and_k<LpSrcOp<FP16>, false>(LpSrcOp<FP16>{a.src_lp, a.scale}, a);
+    return 1;
+}
+#elif FBSR_GROUP == 3
+int FBSR_CAT(dispatch_qat_adamw_, FBSR_FMT)(const CallArgs& a)
+{
+    static_assert(CODE_BYTES == 1, "the weights of Algorithm 1 are 8 bits wide");
+    if (a.src_fmt == BF16) {
+        return by_variant_and_k<QatAdamOp<FMT, BF16>, false>(
+            QatAdamOp<FMT, BF16>{a.dst, a.src_lp, a.m, a.v, a.beta1, a.beta2, a.eps, a.neg_c1, a.c2, a.a1, a.a2, a.neg_lrwd}, a);
+    }
+    if (a.src_fmt == FP16) {
+        return by_variant_and_k<QatAdamOp<FMT, FP16>, false>(
+            QatAdamOp<FMT, FP16>{a.dst, a.src_lp, a.m, a.v, a.beta1, a.beta2, a.eps, a.neg_c1, a.c2, a.a1, a.a2, a.neg_lrwd}, a);
+    }
     return 1;
 }
 #else

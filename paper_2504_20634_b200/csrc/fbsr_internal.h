@@ -6,7 +6,7 @@
 
 namespace fbsr {
 
-enum OpKind { OP_ROUND = 0, OP_ROUND_BITS, OP_ROUND_STATS, OP_SGD, OP_ADAM, OP_ACCUM, OP_ROUND_LP, OP_QAT, OP_ROUND_MX };
+enum OpKind { OP_ROUND = 0, OP_ROUND_BITS, OP_ROUND_STATS, OP_SGD, OP_ADAM, OP_ACCUM, OP_ROUND_LP, OP_QAT, OP_ROUND_MX, OP_QAT_ADAMW };
 
 // Everything an entry point hands to the per-format dispatcher.  Validated by the caller.
 struct CallArgs {
@@ -34,16 +34,18 @@ struct CallArgs {
     float* w; const float* g; float* m; float* v;
     float neg_lr, mu;                                   // SGD-momentum
     float beta1, beta2, eps, neg_c1, c2, a1, a2;        // Adam
+    float neg_lrwd;                                     // OP_QAT_ADAMW: -(lr * weight_decay)
 };
 
 constexpr int MAX_SLOW_GRID = 148 * 8;      // CTAs of the general kernel; also the number of partial slots
 
 // One dispatcher per (format, op group); each lives in its own translation unit
-// (dispatch_lp_* exists for the 8-bit targets only).
+// (dispatch_lp_* and dispatch_qat_adamw_* exist for the 8-bit targets only).
 #define FBSR_DECLARE_DISPATCH(fmt) \
     int dispatch_round_##fmt(const CallArgs&); \
     int dispatch_optim_##fmt(const CallArgs&);\
-    int dispatch_lp_##fmt(const CallArgs&);
+    int dispatch_lp_##fmt(const CallArgs&); \
+    int dispatch_qat_adamw_##fmt(const CallArgs&);
 FBSR_DECLARE_DISPATCH(0) FBSR_DECLARE_DISPATCH(1) FBSR_DECLARE_DISPATCH(2) FBSR_DECLARE_DISPATCH(3) FBSR_DECLARE_DISPATCH(4)
 #undef FBSR_DECLARE_DISPATCH
 

@@ -484,6 +484,69 @@ struct QatOp {
     }
 };
 
+// Algorithm 1 from the gradient on: w16 = value(w8); the AdamW update in binary32 with one rounding per operation,
+// rounded to the 16-bit format (u16); s = RTNE_16(fl32(w16 + u16)); the caller of finish() rounds s to 8 bits.
+//   m' = fma(b1, m, a1 g);  v' = fma(b2, v, (a2 g) g);  d = sqrt(v') c2 + eps;  u32 = fma(-c1, m'/d, -(lr wd) w16)
+template <int WF, int UF>
+struct QatAdamOp {
+    static_assert(Format<WF>::K == 8 && (UF == BF16 || UF == FP16), "8-bit weights, 16-bit gradients and updates");
+    static constexpr int BATCH = ROW_BATCH >= 2 ? ROW_BATCH / 2 : 1, MIN_CTAS = FBSR_MIN_CTAS_ADAM, OCTETS = 1;
+    const void* w8; const void* g16; float* m; float* v;
+    float beta1, beta2, eps, neg_c1, c2, a1, a2, neg_lrwd;
+    struct Regs { uint2 w; uint4 g; F8 m, v; };
+    __device__ __forceinline__ static float widen16(uint32_t code)
+    {
+        return UF == BF16 ? __uint_as_float(code << 16) : __half2float(__ushort_as_half((unsigned short)code));
+    }
+    // round to the 16-bit format, ties to even; a finite value beyond its largest one saturates
+    __device__ __forceinline__ static float round16(float s)
+    {
+        const float m16 = __uint_as_float(Format<UF>::MAXBITS);
+        const float a = fabsf(s);
+        if (a > m16 && a < __uint_as_float(0x7F800000u)) s = copysignf(m16, s);
+        if constexpr (UF == BF16) return __bfloat162float(__float2bfloat16_rn(s));
+        else return __half2float(__float2half_rn(s));
+    }
+    __device__ __forceinline__ float step(float wv, uint32_t gcode, float& mv, float& vv) const
+    {
+        const float gv = widen16(gcode);
+        mv = __fmaf_rn(beta1, mv, __fmul_rn(a1, gv));
+        vv = __fmaf_rn(beta2, vv, __fmul_rn(__fmul_rn(a2, gv), gv));
+        const float d = __fadd_rn(__fmul_rn(__fsqrt_rn(vv), c2), eps);
+        const float u32 = __fmaf_rn(neg_c1, __fdiv_rn(mv, d), __fmul_rn(neg_lrwd, wv));
+        const float u16 = round16(u32);
+        return round16(__fadd_rn(wv, u16));
+    }
+    __device__ __forceinline__ void fetch(size_t elem, Regs& r) const
+    {
+        r.w = *reinterpret_cast<const uint2*>(static_cast<const uint8_t*>(w8) + elem);
+        r.g = *reinterpret_cast<const uint4*>(static_cast<const uint16_t*>(g16) + elem);
+        r.m = load_f8(m + elem); r.v = load_f8(v + elem);
+    }
+    __device__ __forceinline__ void finish(size_t elem, const Regs& r, float (&y)[8]) const
+    {
+        float lo[4], hi[4], mv[8], vv[8];
+        decode4<WF>(r.w.x, lo);
+        decode4<WF>(r.w.y, hi);
+        unpack(r.m, mv); unpack(r.v, vv);
+        const uint32_t gw[4] = {r.g.x, r.g.y, r.g.z, r.g.w};
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+            const uint32_t gcode = (gw[c >> 1] >> ((c & 1) * 16)) & 0xFFFFu;
+            y[c] = step(c < 4 ? lo[c] : hi[c - 4], gcode, mv[c], vv[c]);
+        }
+        store_f8(m + elem, mv); store_f8(v + elem, vv);
+    }
+    __device__ __forceinline__ uint32_t exact_bits(const Regs&, int, float y) const { return arith_bits(y); }
+    __device__ __forceinline__ uint32_t scalar(size_t i) const
+    {
+        float mv = m[i], vv = v[i];
+        const float y = step(decode_element<WF>(static_cast<const uint8_t*>(w8)[i]), static_cast<const uint16_t*>(g16)[i], mv, vv);
+        m[i] = mv; v[i] = vv;
+        return arith_bits(y);
+    }
+};
+
 // ---------------------------------------------------------------------------- packing a row of codes
 // Fast rows: t[] as left by round_row_fast: the code sits in the top K bits of each word (bfloat16 with its sign,
 // the other formats with bit 31 clear and the sign still to be taken from y), so packing is byte selection.

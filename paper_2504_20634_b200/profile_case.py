@@ -17,7 +17,7 @@ from paper_2504_20634_b200 import workloads
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--op", default="round", choices=["round", "sgd", "adam", "accumulate", "stats", "bits", "lp", "mx", "desc"])
+    ap.add_argument("--op", default="round", choices=["round", "sgd", "adam", "accumulate", "stats", "bits", "lp", "mx", "desc", "qat_adamw"])
     ap.add_argument("--src-fmt", default="bf16", help="source format for --op lp")
     ap.add_argument("--fmt", default="bf16")
     ap.add_argument("--variant", default="srf")
@@ -44,6 +44,14 @@ def main():
                                   "b8p4": (8, 4, 8, 0x7E, 0x7F, 0x80, True)}[args.fmt])
         bytes_per_elem = 4 + code_bytes
         run = lambda s: fbsr.fbsr_round_desc(x, desc, args.variant, args.k, seed=1234, out=out)
+    elif args.op == "qat_adamw":
+        # Algorithm 1 fused: 8-bit weights in place, 16-bit gradients, binary32 moments: 20 B/parameter
+        fbsr.fbsr_round(x.mul(2.0 ** -18).clamp_(-3, 3), args.fmt, "rtne", 1, seed=0, out=out)
+        g16 = (torch.randn(n, device=dev) * 1e-2).to(torch.bfloat16 if args.src_fmt == "bf16" else torch.float16).view(torch.uint16)
+        m, v = torch.zeros(n, device=dev), torch.zeros(n, device=dev)
+        bytes_per_elem = 20
+        run = lambda s: fbsr.fbsr_qat_adamw_step(out, g16, m, v, args.fmt, args.src_fmt, args.variant, args.k, s, 0,
+                                                 1e-3, 0.9, 0.95, 1e-8, 0.1, s + 1)
     elif args.op == "lp":
         codes = workloads.lp_sweep(n, args.src_fmt, device=dev)
         bytes_per_elem = 2 + code_bytes
