@@ -349,7 +349,21 @@ def main():
         b.record(stream)
         torch.cuda.synchronize()
         extras["qat_update_b8p4_bf16_src_k3_GBps"] = round(4.0 * n_local / (a.elapsed_time(b) / 10 * 1e-3) / 1e9, 1)
-        del codes16, w8, upd
+        # one whole iteration of Algorithm 1, fused (20 B/parameter): Binary8P4 weights, bf16 gradients, 3 random bits
+        grad16 = upd
+        m_ = torch.zeros(n_local, device=dev)
+        v_ = torch.zeros(n_local, device=dev)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        fbsr.fbsr_qat_adamw_step(w8, grad16, m_, v_, "b8p4", "bf16", "src", 3, 1, 0, 1e-3, 0.9, 0.95, 1e-8, 0.1, 1)
+        a.record(stream)
+        for s_ in range(10):
+            fbsr.fbsr_qat_adamw_step(w8, grad16, m_, v_, "b8p4", "bf16", "src", 3, 2 + s_, 0, 1e-3, 0.9, 0.95, 1e-8, 0.1, 2 + s_)
+        b.record(stream)
+        torch.cuda.synchronize()
+        ms_ = a.elapsed_time(b) / 10
+        extras["qat_adamw_step_b8p4_bf16_src_k3"] = {"Gparam/s": round(n_local / (ms_ * 1e-3) / 1e9, 2),
+                                                      "GB/s": round(20.0 * n_local / (ms_ * 1e-3) / 1e9, 1)}
+        del codes16, w8, upd, grad16, m_, v_
         # fused optimizer step on the 32-block parameter list (22 B/param SGD-momentum, 30 B/param Adam)
         try:
             n_p = workloads.optimizer_param_count(32)

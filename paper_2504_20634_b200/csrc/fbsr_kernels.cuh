@@ -38,6 +38,12 @@ namespace fbsr {
 #ifndef FBSR_MIN_CTAS_SGD
 #define FBSR_MIN_CTAS_SGD 2
 #endif
+#ifndef FBSR_QATADAM_BATCH
+#define FBSR_QATADAM_BATCH 1      // rows of loads in flight per warp for the fused Algorithm-1 step; measured with
+#endif
+#ifndef FBSR_QATADAM_MIN_CTAS
+#define FBSR_QATADAM_MIN_CTAS 4   // (1, 4): 6.4-6.6 TB/s; (2, 3): 6.3-6.7; (2, 2): 5.6-5.8; (1, 6): 6.0-6.1
+#endif
 #ifndef FBSR_MIN_CTAS_ADAM
 #define FBSR_MIN_CTAS_ADAM 2
 #endif
@@ -490,7 +496,7 @@ struct QatOp {
 template <int WF, int UF>
 struct QatAdamOp {
     static_assert(Format<WF>::K == 8 && (UF == BF16 || UF == FP16), "8-bit weights, 16-bit gradients and updates");
-    static constexpr int BATCH = ROW_BATCH >= 2 ? ROW_BATCH / 2 : 1, MIN_CTAS = FBSR_MIN_CTAS_ADAM, OCTETS = 1;
+    static constexpr int BATCH = FBSR_QATADAM_BATCH, MIN_CTAS = FBSR_QATADAM_MIN_CTAS, OCTETS = 1;
     const void* w8; const void* g16; float* m; float* v;
     float beta1, beta2, eps, neg_c1, c2, a1, a2, neg_lrwd;
     struct Regs { uint2 w; uint4 g; F8 m, v; };
