@@ -307,7 +307,40 @@ __device__ __forceinline__ bool round_row_fast(const float (&y)[8], const Draws8
     constexpr int EFF = R::deterministic ? VAR : (R::ALL_BITS || (FMT == BF16 && N == 16)) ? SRFF : VAR;
     constexpr int POS = R::deterministic ? SH0 : SH0 - N;     // where the draw (or the half step) is added
     float flag = 0.0f;
-    if constexpr (!R::one_regime) {
+    if constexpr (!R::one_regime && N >= SH0) {
+        // Draws at least as wide as the excess bits of a normal result (binary16 with N = 13..16).  Both candidates
+        // are formed with the code in the top K bits, and the draw enters both as the same term
+        // D = n 2^(W - N), W = 32 - K:
+        //   |y| >= 2^emin: every variant is exact SR on the sh0 excess bits: (pattern << L) + D; the bits of D below
+        //                  the pattern's lowest bit meet zeros and cannot carry;
+        //   |y| <  2^emin: floor(sigma~ + n 2^-N) is the top K bits of floor(sigma~ 2^W) + D (SRFF); SRF adds half a
+        //                  step more (at N = W one position finer, then one shift); SRC converts sigma~ 2^N to
+        //                  nearest-even first.
+        static_assert(FMT != BF16 && F::K == 16, "only binary16 has draws wider than its excess bits");
+        constexpr int W = 32 - F::K, L = W - SH0;                                       // 16, 3
+        static_assert(N <= W && L >= 0, "the draw fits under the code");
+        const float rescale = __uint_as_float((uint32_t)(128 - F::EMINB) << 23);        // 2^(1 - EMINB)
+        const float min_normal = __uint_as_float((uint32_t)F::EMINB << 23);             // 2^emin
+        // sigma~ 2^X = |y| 2^(X + P - 1 - emin); emin = EMINB - 127
+        constexpr int X = VAR == SRC ? N : (VAR == SRF && N == W) ? W + 1 : W;
+        const float to_steps = __uint_as_float((uint32_t)(X + F::P - 1 + 254 - F::EMINB) << 23);
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+            const float a = fabsf(y[c]);
+            flag = __fmaf_rn(y[c], 0.0f, flag);
+            const uint32_t D = d.template at<W - N>(c);
+            const uint32_t u = min(__float_as_uint(__fmul_rz(a, rescale)), F::MAXCODE << SH0);
+            const uint32_t hi = u * (1u << L) + D;
+            const float steps = __fmul_rn(a, to_steps);                                 // exact below 2^emin
+            uint32_t lo;
+            if constexpr (VAR == SRFF) lo = __float2uint_rz(steps) + D;
+            else if constexpr (VAR == SRF && N < W) lo = __float2uint_rz(steps) + D + (1u << (W - N - 1));
+            else if constexpr (VAR == SRF) lo = (__float2uint_rz(steps) + 2u * D + 1u) >> 1;
+            else lo = __float2uint_rn(steps) * (1u << (W - N)) + D;
+            t[c] = a < min_normal ? lo : hi;
+        }
+        return flag != flag;
+    } else if constexpr (!R::one_regime) {
         static_assert(FMT != BF16 && N >= SH0 - 1, "two-regime form is for draws about as wide as the excess bits");
         const float rescale = __uint_as_float((uint32_t)(128 - F::EMINB) << 23);        // 2^(1 - EMINB)
         const float min_normal = __uint_as_float((uint32_t)F::EMINB << 23);             // 2^emin

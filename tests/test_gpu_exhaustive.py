@@ -10,7 +10,7 @@ import torch
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("fmt,variant,k", [("bf16", "src", 5), ("e4m3", "srf", 3), ("fp16", "src", 13)])
+@pytest.mark.parametrize("fmt,variant,k", [("bf16", "src", 5), ("e4m3", "srf", 3), ("fp16", "src", 13), ("b8p4", "src", 3)])
 def test_all_binary32_patterns(fmt, variant, k):
     import paper_2504_20634_b200 as fbsr
     from oracle import capi
