@@ -35,6 +35,11 @@
  * (b lo, b hi, stream, 0), key (seed lo, seed hi), output word (g mod E) / dpw,
  * field g mod dpw counted from the low bits.
  *
+ * Parity unpinned by the paper (the library's own definitions, pinned only by the means named): the policy for
+ * special and out-of-range values (torch's casts); the optimizer arithmetic of the SGD / Adam / Algorithm-1 steps
+ * (exact-rational replay, torch.optim); the block-scale recipe (numpy's frexp); Binary8P4's bias, M and special
+ * patterns, which the paper does not print (the P3109 report's values; torch's float8_e4m3fnuz for all but 0x7F).
+ *
  * Build: gcc -O2 -std=c11 -ffp-contract=off -fno-fast-math -shared -fPIC
  * (no contraction: every binary32 operation below rounds exactly once).
  */
