@@ -450,16 +450,21 @@ struct QatOp {
     struct Regs { uint32_t w[4]; uint32_t u[8]; };
     __device__ __forceinline__ static float sum16(uint32_t wcode, uint32_t ucode)
     {
-        return sum16v(decode_element<WF>(wcode), ucode);
+        return sum16v<true>(decode_element<WF>(wcode), ucode);
     }
+    // EXACT: round to the 16-bit format with ties to even, a finite sum beyond its largest value saturating.
+    // !EXACT: the plain hardware conversion, which turns such a sum into an infinity instead; the row is then
+    // flagged like any row holding Inf or NaN and redone through exact_bits(), so the check is paid only there.
+    template <bool EXACT>
     __device__ __forceinline__ static float sum16v(float wv, uint32_t ucode)
     {
         const float uv = UF == BF16 ? __uint_as_float(ucode << 16) : __half2float(__ushort_as_half((unsigned short)ucode));
         float s = __fadd_rn(wv, uv);
-        // round to the 16-bit format, ties to even; a finite sum beyond its largest value saturates
-        const float m16 = __uint_as_float(Format<UF>::MAXBITS);
-        const float a = fabsf(s);
-        if (a > m16 && a < __uint_as_float(0x7F800000u)) s = copysignf(m16, s);
+        if constexpr (EXACT) {
+            const float m16 = __uint_as_float(Format<UF>::MAXBITS);
+            const float a = fabsf(s);
+            if (a > m16 && a < __uint_as_float(0x7F800000u)) s = copysignf(m16, s);
+        }
         if constexpr (UF == BF16) return __bfloat162float(__float2bfloat16_rn(s));
         else return __half2float(__float2half_rn(s));
     }
@@ -480,10 +485,15 @@ struct QatOp {
 #pragma unroll
         for (int c = 0; c < 8; ++c) {
             const uint32_t ucode = (r.u[4 * o + (c >> 1)] >> ((c & 1) * 16)) & 0xFFFFu;
-            y[c] = sum16v(c < 4 ? lo[c] : hi[c - 4], ucode);
+            y[c] = sum16v<false>(c < 4 ? lo[c] : hi[c - 4], ucode);
         }
     }
-    __device__ __forceinline__ uint32_t exact_bits(const Regs&, int, int, float y) const { return arith_bits(y); }
+    __device__ __forceinline__ uint32_t exact_bits(const Regs& r, int o, int c, float) const
+    {
+        const uint32_t wcode = (r.w[2 * o + (c >> 2)] >> ((c & 3) * 8)) & 0xFFu;
+        const uint32_t ucode = (r.u[4 * o + (c >> 1)] >> ((c & 1) * 16)) & 0xFFFFu;
+        return arith_bits(sum16(wcode, ucode));
+    }
     __device__ __forceinline__ uint32_t scalar(size_t i) const
     {
         return arith_bits(sum16(static_cast<const uint8_t*>(w8)[i], static_cast<const uint16_t*>(u16)[i]));
@@ -504,15 +514,21 @@ struct QatAdamOp {
     {
         return UF == BF16 ? __uint_as_float(code << 16) : __half2float(__ushort_as_half((unsigned short)code));
     }
-    // round to the 16-bit format, ties to even; a finite value beyond its largest one saturates
+    // EXACT: round to the 16-bit format, ties to even, a finite value beyond its largest one saturating.
+    // !EXACT: the plain hardware conversion, which gives an infinity there; that infinity survives to the result
+    // (w + Inf is Inf or NaN), the row is flagged and redone through exact_bits(), as for QatOp.
+    template <bool EXACT>
     __device__ __forceinline__ static float round16(float s)
     {
-        const float m16 = __uint_as_float(Format<UF>::MAXBITS);
-        const float a = fabsf(s);
-        if (a > m16 && a < __uint_as_float(0x7F800000u)) s = copysignf(m16, s);
+        if constexpr (EXACT) {
+            const float m16 = __uint_as_float(Format<UF>::MAXBITS);
+            const float a = fabsf(s);
+            if (a > m16 && a < __uint_as_float(0x7F800000u)) s = copysignf(m16, s);
+        }
         if constexpr (UF == BF16) return __bfloat162float(__float2bfloat16_rn(s));
         else return __half2float(__float2half_rn(s));
     }
+    template <bool EXACT>
     __device__ __forceinline__ float step(float wv, uint32_t gcode, float& mv, float& vv) const
     {
         const float gv = widen16(gcode);
@@ -520,8 +536,8 @@ struct QatAdamOp {
         vv = __fmaf_rn(beta2, vv, __fmul_rn(__fmul_rn(a2, gv), gv));
         const float d = __fadd_rn(__fmul_rn(__fsqrt_rn(vv), c2), eps);
         const float u32 = __fmaf_rn(neg_c1, __fdiv_rn(mv, d), __fmul_rn(neg_lrwd, wv));
-        const float u16 = round16(u32);
-        return round16(__fadd_rn(wv, u16));
+        const float u16 = round16<EXACT>(u32);
+        return round16<EXACT>(__fadd_rn(wv, u16));
     }
     __device__ __forceinline__ void fetch(size_t elem, Regs& r) const
     {
@@ -539,15 +555,25 @@ struct QatAdamOp {
 #pragma unroll
         for (int c = 0; c < 8; ++c) {
             const uint32_t gcode = (gw[c >> 1] >> ((c & 1) * 16)) & 0xFFFFu;
-            y[c] = step(c < 4 ? lo[c] : hi[c - 4], gcode, mv[c], vv[c]);
+            y[c] = step<false>(c < 4 ? lo[c] : hi[c - 4], gcode, mv[c], vv[c]);
         }
         store_f8(m + elem, mv); store_f8(v + elem, vv);
     }
-    __device__ __forceinline__ uint32_t exact_bits(const Regs&, int, float y) const { return arith_bits(y); }
+    // the element again, from the values fetched before the update, with the saturating conversions
+    __device__ __forceinline__ uint32_t exact_bits(const Regs& r, int c, float) const
+    {
+        float mo[8], vo[8];
+        unpack(r.m, mo); unpack(r.v, vo);
+        const uint32_t wcode = ((c < 4 ? r.w.x : r.w.y) >> ((c & 3) * 8)) & 0xFFu;
+        const uint32_t gw[4] = {r.g.x, r.g.y, r.g.z, r.g.w};
+        const uint32_t gcode = (gw[c >> 1] >> ((c & 1) * 16)) & 0xFFFFu;
+        float mv = mo[c], vv = vo[c];
+        return arith_bits(step<true>(decode_element<WF>(wcode), gcode, mv, vv));
+    }
     __device__ __forceinline__ uint32_t scalar(size_t i) const
     {
         float mv = m[i], vv = v[i];
-        const float y = step(decode_element<WF>(static_cast<const uint8_t*>(w8)[i]), static_cast<const uint16_t*>(g16)[i], mv, vv);
+        const float y = step<true>(decode_element<WF>(static_cast<const uint8_t*>(w8)[i]), static_cast<const uint16_t*>(g16)[i], mv, vv);
         m[i] = mv; v[i] = vv;
         return arith_bits(y);
     }

@@ -62,6 +62,10 @@ def test_qat_update(w_fmt, u_fmt):
     dt = torch.bfloat16 if u_fmt == "bf16" else torch.float16
     small16 = torch.from_numpy(small).to(dt).view(torch.int16).numpy().view(np.uint16)
     u16[: n - 500] = small16[: n - 500]
+    # finite sums beyond the 16-bit format's largest value (they saturate; they do not become infinities):
+    # the largest finite update code next to weights of the same sign
+    top = 0x7F7F if u_fmt == "bf16" else 0x7BFF
+    u16[100:164] = np.where(w8[100:164] & 0x80, 0x8000 | top, top).astype(np.uint16)
     for variant, k in (("srff", 3), ("srf", 3), ("src", 3), ("src", 8), ("rtne", 1), ("srf", 16)):
         wd = gu.from_np_codes(w8)
         fbsr.fbsr_qat_update(wd, gu.from_np_codes(u16), w_fmt, u_fmt, variant, k, seed=4, offset=11)

@@ -58,6 +58,27 @@ def test_parity_every_variant(w_fmt, g_fmt):
         assert same_state(md, m1) and same_state(vd, v1)
 
 
+def test_updates_beyond_the_16_bit_range_saturate():
+    """A learning rate so large that the update overflows binary16: u16 saturates at -+65504 (it does not become an
+    infinity), and so does the 16-bit sum."""
+    rng = np.random.default_rng(79)
+    for w_fmt in ("e5m2", "b8p4", "e4m3"):
+        n = 6 * 1536 + 11
+        w8, g16, m, v = make_case(rng, w_fmt, "fp16", n, specials=False)
+        for lr in (1e6, 3e4):
+            wd, gd = gu.from_np_codes(w8), gu.from_np_codes(g16)
+            md, vd = torch.from_numpy(m).cuda(), torch.from_numpy(v).cuda()
+            kw = dict(lr=lr, beta1=0.9, beta2=0.95, eps=1e-8, weight_decay=0.1)
+            fbsr.fbsr_qat_adamw_step(wd, gd, md, vd, w_fmt, "fp16", "srf", 5, seed=1, offset=0, step=1, **kw)
+            w1, m1, v1 = w8.copy(), m.copy(), v.copy()
+            capi.qat_adamw_step(w1, g16, m1, v1, w_fmt, "fp16", "srf", 5, seed=1, offset=0, step=1, **kw)
+            gu.assert_codes_equal(wd, w1, "%s lr=%g" % (w_fmt, lr))
+            assert same_state(md, m1) and same_state(vd, v1)
+            # most weights end at the largest finite value, none at an infinity
+            top8 = {"e5m2": 0x7B, "b8p4": 0x7E, "e4m3": 0x7E}[w_fmt]
+            assert not np.any((w1 & 0x7F) == 0x7F) and (lr < 1e6 or np.mean((w1 & 0x7F) == top8) > 0.5)
+
+
 def test_unaligned_pointers_offsets_and_small_sizes():
     rng = np.random.default_rng(73)
     for n in (0, 1, 7, 255, 3000):
