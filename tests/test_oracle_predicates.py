@@ -212,3 +212,22 @@ def test_array_call_is_elementwise_with_global_index():
         assert np.array_equal(whole, capi.fbsr_round_bits(x, "fp16", "srf", k, words))
         one_by_one = [capi.round_one(x[i], "fp16", "srf", k, capi.draw(77, i, k))[0] for i in range(50)]
         assert list(whole[:50]) == one_by_one
+
+
+@pytest.mark.parametrize("fmt", FMTS + ("b8p4",))
+@pytest.mark.parametrize("variant", VARIANTS + ("rtne", "rta", "rto"))
+def test_rounding_is_monotone_in_the_magnitude(fmt, variant):
+    """For a fixed draw, floor(sigma~) + [R] never decreases when the value grows (each predicate is monotone in
+    delta~, and a larger floor outweighs any predicate), and codes of positive values are ordered like the values:
+    sorted magnitudes must give non-decreasing codes, through binade changes, the subnormal range and saturation."""
+    rng = np.random.default_rng(97)
+    lo, hi = {"bf16": (-126, 127), "fp16": (-30, 17), "e4m3": (-14, 10), "e5m2": (-22, 17), "b8p4": (-15, 9)}[fmt]
+    mags = np.sort(bits_f32(random_f32(rng, 30000, lo, hi) & np.uint32(0x7FFFFFFF)))
+    # and a dense run of consecutive binary32 values across a rounding boundary
+    mags = np.concatenate([mags, bits_f32(np.arange(0x3F7FFF00, 0x3F800100, dtype=np.uint32))])
+    mags = np.sort(mags)
+    for k in (1, 3, 7, 16):
+        for n in (0, (1 << k) // 3, (1 << k) - 1):
+            words_n = n
+            codes = np.array([capi.round_one(y, fmt, variant, k, words_n)[0] for y in mags[::7]], dtype=np.int64)
+            assert np.all(np.diff(codes) >= 0), (fmt, variant, k, n)
