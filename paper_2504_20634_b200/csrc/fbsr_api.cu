@@ -148,7 +148,7 @@ int fbsr_round_stats(const float* src, void* dst, size_t n, int fmt, int variant
 
 }  // extern "C"
 
-// Scratch of the no-allocation statistics entry point: one slot per CTA of the general kernel.
+// Scratch of the no-allocation statistics entry point: one slot per CTA of the statistics kernels.
 // In host code this name is only a handle for cudaGetSymbolAddress, never a device address.
 static __device__ __align__(256) unsigned char g_noalloc_stats_scratch[FBSR_NOALLOC_SCRATCH_BYTES];
 static_assert(FBSR_NOALLOC_SCRATCH_BYTES == MAX_SLOW_GRID * sizeof(fbsr_stats), "scratch must hold one partial per CTA");

@@ -169,23 +169,75 @@ int by_variant_and_k(const Op& op, const CallArgs& a)
 
 #if FBSR_GROUP == 0
 namespace {
-template <int K>
-void launch_stats_rows(const CallArgs& a, uint64_t n_rows, int n_ctas)
+// Statistics: the head of the call (up to the first tile boundary of the draw stream) and the ragged end go to the
+// general kernel, whole tiles to the tiled statistics kernel; every CTA leaves one partial in the workspace (tiles
+// first, then head, then end) and stats_finalize_kernel adds them in that order.
+constexpr int STATS_EDGE_SLOTS = 8;                                    // per edge; an edge is less than one tile
+constexpr int STATS_TILE_GRID = MAX_SLOW_GRID - 2 * STATS_EDGE_SLOTS;  // CTAs (and partial slots) of the tiled kernel
+
+template <int VAR, int K>
+int run_stats(const CallArgs& a)
 {
-    stats_row_kernel<FMT, K><<<(unsigned)n_ctas, CTA_THREADS, 0, a.stream>>>(
-        a.src, a.scale, a.dst, n_rows, a.offset, a.variant, (uint32_t)a.seed, (uint32_t)(a.seed >> 32), a.group_size,
-        a.gsum_e, a.gsum_e2, static_cast<StatsAcc*>(a.partials));
+    const RoundOp op{a.src, a.scale};
+    StatsAcc* slots = static_cast<StatsAcc*>(a.partials);
+    int n_slots = 0;
+    const Plan p = a.ovf_ieee ? Plan{0, 0, 0} : make_plan<RoundOp, K, false>(op, a);
+    if (p.n_tiles > 0) {
+        using T = Tile<K, 1>;
+        const uint64_t want = (p.n_tiles + WARPS_PER_CTA - 1) / WARPS_PER_CTA;
+        const unsigned grid = (unsigned)(want < (uint64_t)STATS_TILE_GRID ? want : (uint64_t)STATS_TILE_GRID);
+        stats_tile_kernel<FMT, VAR, K><<<grid, CTA_THREADS, 0, a.stream>>>(
+            a.src + p.head, a.scale, static_cast<char*>(a.dst) + p.head * CODE_BYTES, p.n_tiles, p.head,
+            (a.offset + p.head) / T::E, (uint32_t)a.seed, (uint32_t)(a.seed >> 32), a.group_size, a.gsum_e, a.gsum_e2,
+            slots);
+        count_launch();
+        n_slots = (int)grid;
+        CallArgs edge = a;
+        int used = 0;
+        edge.partials = slots + n_slots;
+        launch_generic<RoundOp, false, true>(op, edge, 0, p.head, &used);
+        n_slots += used;
+        edge.partials = slots + n_slots;
+        launch_generic<RoundOp, false, true>(op, edge, p.tail_begin, a.n, &used);
+        n_slots += used;
+    } else {
+        launch_generic<RoundOp, false, true>(op, a, 0, a.n, &n_slots);
+    }
+    stats_finalize_kernel<<<1, CTA_THREADS, 0, a.stream>>>(slots, n_slots, static_cast<StatsAcc*>(a.total));
+    count_launch();
+    return 0;
 }
-template <int... Ks>
-void stats_rows_dispatch(const CallArgs& a, uint64_t n_rows, int n_ctas, std::integer_sequence<int, Ks...>)
+
+template <int VAR>
+int stats_by_k(const CallArgs& a)
 {
-    using Fn = void (*)(const CallArgs&, uint64_t, int);
-    static constexpr Fn table[16] = {&launch_stats_rows<Ks + 1>...};
-    table[a.k - 1](a, n_rows, n_ctas);
+    switch (a.k) {
+    case 1: return run_stats<VAR, 1>(a);
+    case 2: return run_stats<VAR, 2>(a);
+    case 3: return run_stats<VAR, 3>(a);
+    case 4: return run_stats<VAR, 4>(a);
+    case 5: return run_stats<VAR, 5>(a);
+    case 6: return run_stats<VAR, 6>(a);
+    case 7: return run_stats<VAR, 7>(a);
+    case 8: return run_stats<VAR, 8>(a);
+    case 9: return run_stats<VAR, 9>(a);
+    case 10: return run_stats<VAR, 10>(a);
+    case 11: return run_stats<VAR, 11>(a);
+    case 12: return run_stats<VAR, 12>(a);
+    case 13: return run_stats<VAR, 13>(a);
+    case 14: return run_stats<VAR, 14>(a);
+    case 15: return run_stats<VAR, 15>(a);
+    case 16: return run_stats<VAR, 16>(a);
+    default: return 1;
+    }
 }
-inline void stats_rows_by_k(const CallArgs& a, uint64_t n_rows, int n_ctas)
+
+int stats_by_variant_and_k(const CallArgs& a)
 {
-    stats_rows_dispatch(a, n_rows, n_ctas, std::make_integer_sequence<int, 16>{});
+    if (a.variant == RTNE) return run_stats<RTNE, 16>(a);
+    if (a.variant == RTA) return run_stats<RTA, 16>(a);
+    if (a.variant == RTO) return run_stats<RTO, 16>(a);
+    return a.variant == SRFF ? stats_by_k<SRFF>(a) : a.variant == SRF ? stats_by_k<SRF>(a) : stats_by_k<SRC>(a);
 }
 }  // namespace
 
@@ -196,29 +248,7 @@ int FBSR_CAT(dispatch_round_, FBSR_FMT)(const CallArgs& a)
     case OP_ROUND: return by_variant_and_k<RoundOp, false>(op, a);
     case OP_ROUND_BITS: return by_variant_and_k<RoundOp, true>(op, a);
     case OP_ROUND_MX: return by_variant_and_k<MxOp<FMT>, false>(MxOp<FMT>{a.src, a.scales, a.n}, a);
-    case OP_ROUND_STATS: {
-        // Whole rows of 256 elements go to the row kernel when the pointers allow vector access, the rest to
-        // the general kernel; each CTA leaves one partial in the workspace and they are summed in a fixed order.
-        int n_ctas = 0;
-        uint64_t n_rows = 0;
-        if (!a.ovf_ieee && aligned(a.src, 32) && aligned(a.dst, CODE_BYTES == 2 ? 16 : 8)) n_rows = a.n / ROW_ELEMS;
-        if (n_rows > 0) {
-            const uint64_t want = (n_rows + WARPS_PER_CTA - 1) / WARPS_PER_CTA;
-            const uint64_t cap = MAX_SLOW_GRID - 8;                 // the last slots belong to the ragged end
-            n_ctas = (int)(want < cap ? want : cap);
-            stats_rows_by_k(a, n_rows, n_ctas);
-            count_launch();
-        }
-        CallArgs rest = a;
-        rest.partials = static_cast<StatsAcc*>(a.partials) + n_ctas;
-        int rest_ctas = 0;
-        launch_generic<RoundOp, false, true>(op, rest, n_rows * ROW_ELEMS, a.n, &rest_ctas);
-        n_ctas += rest_ctas;
-        stats_finalize_kernel<<<1, CTA_THREADS, 0, a.stream>>>(static_cast<const StatsAcc*>(a.partials), n_ctas,
-                                                               static_cast<StatsAcc*>(a.total));
-        count_launch();
-        return 0;
-    }
+    case OP_ROUND_STATS: return stats_by_variant_and_k(a);
     default: return 1;
     }
 }

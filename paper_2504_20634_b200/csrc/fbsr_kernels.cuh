@@ -855,73 +855,156 @@ generic_kernel(const Op op, void* __restrict__ dst, const uint64_t i_begin, cons
     }
 }
 
-// Statistics on aligned rows: a warp takes rows of 256 elements (one 256-bit load and one packed store per
-// lane), every lane computes the one or two generator calls that cover its 8 elements, rounds them with the
-// element-wise integer rounder and accumulates e = up - delta in binary64.  Any `offset` is served, because
-// the draws are located from the global index; only the pointers must be vector-aligned.
-template <int FMT, int K>
-__global__ void __launch_bounds__(CTA_THREADS)
-stats_row_kernel(const float* __restrict__ src, const float scale, void* __restrict__ dst, const uint64_t n_rows,
-                 const uint64_t offset, const int variant, const uint32_t k0, const uint32_t k1,
-                 const uint64_t group_size, double* __restrict__ gsum_e, double* __restrict__ gsum_e2,
-                 StatsAcc* __restrict__ partials)
+// Statistics of one element from its value and the magnitude of the code it was given (the draw is not needed):
+// floor(sigma~) and delta~ come from the decomposition of Eq. (2)-(3), up = code - code of the floor, e = up - delta~.
+// Returns true and sets e and up for an SR-rounded element; the others are only counted.
+template <int FMT>
+__device__ __forceinline__ bool stats_element(const uint32_t ybits, const uint32_t code_mag, StatsAcc& acc, double& e,
+                                              uint32_t& up)
 {
-    using T = Tile<K>;
-    static_assert(T::E >= 8, "a lane's 8 elements span at most two generator calls");
+    using F = Format<FMT>;
+    constexpr int P = F::P;
+    const uint32_t mag = ybits & 0x7FFFFFFFu;
+    if (mag > F::MAXBITS) {
+        if (mag > 0x7F800000u) acc.n_nan += 1;
+        else if (mag == 0x7F800000u) acc.n_inf += 1;
+        else acc.n_sat += 1;
+        return false;
+    }
+    uint32_t r;
+    int sh;
+    if constexpr (FMT == BF16) {
+        sh = 16;                                             // same exponent range as binary32: the low half is delta~
+        r = mag & 0xFFFFu;
+        up = code_mag - (mag >> 16);
+    } else {
+        const uint32_t e32 = mag >> 23;
+        const uint32_t m = (mag & 0x7FFFFFu) | (e32 ? 0x800000u : 0u);
+        const int eb = max((int)e32, 1);
+        const int te = max(eb, F::EMINB);
+        sh = (24 - P) + (te - eb);
+        const uint32_t fl = sh < 32 ? m >> sh : 0u;
+        r = sh < 32 ? (m & ((1u << sh) - 1u)) : m;
+        up = code_mag - (((uint32_t)(te - F::EMINB) << (P - 1)) + fl);
+    }
+    const double delta = (double)r * __hiloint2double((1023 - sh) << 20, 0);     // r 2^-sh, exact
+    e = (up ? 1.0 : 0.0) - delta;
+    return true;
+}
+
+// Statistics on whole tiles: the rounding of the bandwidth kernel (generator calls shared through the warp's
+// buffer, row rounder, packed stores) followed, per element, by stats_element() on the value and its code.
+// A capped grid walks the tiles with a fixed stride, so each thread adds its elements in a fixed order and
+// leaves one partial per CTA: the totals are reproducible bit for bit.
+// first_index: index within the call of element 0 (for the group sums).
+template <int FMT, int VAR, int K>
+__global__ void __launch_bounds__(CTA_THREADS, 3)
+stats_tile_kernel(const float* __restrict__ src, const float scale, void* __restrict__ dst, const uint64_t n_tiles,
+                  const uint64_t first_index, const uint64_t call0, const uint32_t k0, const uint32_t k1,
+                  const uint64_t group_size, double* __restrict__ gsum_e, double* __restrict__ gsum_e2,
+                  StatsAcc* __restrict__ partials)
+{
+    using T = Tile<K, 1>;
+    using F = Format<FMT>;
+    constexpr bool DRAWS = VAR < RTNE;
+    constexpr bool OWN_CALL = T::DPW == 2;
+    constexpr int ROWS = T::ELEMS / ROW_ELEMS;
+    constexpr int WPO = WordsPerOctet<FMT>::value;
+    constexpr uint32_t MAG = (1u << (F::K - 1)) - 1u;
+    __shared__ __align__(16) uint32_t wordbuf[WARPS_PER_CTA][OWN_CALL ? 4 : T::WORDS + 4];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const bool draws = variant < RTNE;
+    uint32_t* wb = wordbuf[warp];
     StatsAcc acc;
     stats_zero(acc);
-    for (uint64_t row = (uint64_t)blockIdx.x * WARPS_PER_CTA + warp; row < n_rows;
-         row += (uint64_t)gridDim.x * WARPS_PER_CTA) {
-        const uint64_t i0 = row * ROW_ELEMS + lane * 8;
-        float x[8];
-        unpack(load_f8_stream(src + i0), x);
-        const uint64_t g0 = offset + i0, call = g0 / T::E;
-        const uint32_t j0 = (uint32_t)(g0 - call * T::E);
-        uint4 a = make_uint4(0u, 0u, 0u, 0u), b = a;
-        if (draws) {
-            a = philox_block(call, k0, k1);
-            b = (j0 + 7 >= (uint32_t)T::E) ? philox_block(call + 1, k0, k1) : a;
-        }
-        uint64_t grp = 0, grp_end = ~0ull;
-        double ge = 0.0, ge2 = 0.0;
-        if (group_size) { grp = i0 / group_size; grp_end = (grp + 1) * group_size; }
-        uint32_t codes[8];
+
+    for (uint64_t tile = (uint64_t)blockIdx.x * WARPS_PER_CTA + warp; tile < n_tiles;
+         tile += (uint64_t)gridDim.x * WARPS_PER_CTA) {
+        const size_t e0 = (size_t)tile * T::ELEMS;
+        const uint64_t tile_call0 = call0 + tile * T::CALLS;
+        // rows are loaded two at a time: the statistics need the registers that deeper prefetching would take
+        constexpr int BATCH = 2;
+        F8 regs[BATCH];
 #pragma unroll
-        for (int c = 0; c < 8; ++c) {
-            uint32_t j = j0 + c;
-            const uint4 o = j < (uint32_t)T::E ? a : b;
-            j = j < (uint32_t)T::E ? j : j - T::E;
-            const uint32_t ws = j / T::DPW;
-            const uint32_t word = ws == 0 ? o.x : ws == 1 ? o.y : ws == 2 ? o.z : o.w;
-            const uint32_t n = (word >> ((j % T::DPW) * K)) & T::MASK;
-            const uint32_t y = scaled_bits(x[c], scale);
-            ElementInfo info;
-            codes[c] = round_core<FMT, true>(y, n, variant, K, &info);
-            if (info.kind == 0) {
-                const double e = (double)info.up - info.delta, e2 = e * e;
-                acc.n_finite += 1; acc.n_up += (unsigned)info.up;
-                acc.sum_e += e; acc.sum_e2 += e2;
-                acc.sum_signed_e += (y >> 31) ? -e : e;
-                acc.sum_abs_e += fabs(e);
-                if (group_size) {
-                    while (i0 + c >= grp_end) {               // this element starts a later group: flush
-                        if (ge != 0.0 || ge2 != 0.0) { atomicAdd(gsum_e + grp, ge); atomicAdd(gsum_e2 + grp, ge2); }
-                        ge = 0.0; ge2 = 0.0;
-                        grp = (i0 + c) / group_size; grp_end = (grp + 1) * group_size;
-                    }
-                    ge += e; ge2 += e2;
+        for (int j = 0; j < BATCH; ++j) regs[j] = load_f8_stream(src + e0 + j * ROW_ELEMS + lane * 8);
+        if constexpr (DRAWS && !OWN_CALL) {
+#pragma unroll
+            for (int j = 0; j < (T::CALLS + 31) / 32; ++j) {
+                const int c = j * 32 + lane;
+                if (T::CALLS % 32 == 0 || c < T::CALLS)
+                    *reinterpret_cast<uint4*>(wb + 4 * c) = philox_block(tile_call0 + c, k0, k1);
+            }
+            __syncwarp();
+        }
+#pragma unroll
+        for (int j = 0; j < ROWS; ++j) {
+            const int p0 = j * ROW_ELEMS + lane * 8;
+            float x[8], y[8];
+            unpack(regs[j % BATCH], x);
+            if (j + BATCH < ROWS) regs[j % BATCH] = load_f8_stream(src + e0 + (j + BATCH) * ROW_ELEMS + lane * 8);
+#pragma unroll
+            for (int c = 0; c < 8; ++c) y[c] = __fmul_rn(x[c], scale);
+            Draws8<K> d;
+            if constexpr (!DRAWS) {
+            } else if constexpr (OWN_CALL) {
+                d.from_call(philox_block(tile_call0 + p0 / 8, k0, k1));
+            } else {
+                d.from_stream(wb, p0);
+            }
+            uint32_t t[8], codes[8], packed[WPO];
+            const bool redo = round_row_fast<FMT, VAR, K>(y, d, t);
+            if (!redo) {
+                pack_row_fast<FMT>(t, y, packed);
+#pragma unroll
+                for (int c = 0; c < 8; ++c) codes[c] = (t[c] >> (32 - F::K)) & MAG;
+            } else {
+#pragma unroll
+                for (int c = 0; c < 8; ++c) {
+                    const uint32_t bits = y[c] != y[c] ? __float_as_uint(x[c]) : __float_as_uint(y[c]);   // a NaN keeps the input's sign
+                    codes[c] = round_core<FMT, false>(bits, d.template at<0>(c), VAR, K, nullptr);
                 }
-            } else if (info.kind == 1) acc.n_nan += 1;
-            else if (info.kind == 2) acc.n_inf += 1;
-            else acc.n_sat += 1;
+                pack_codes8<FMT>(codes, packed);
+#pragma unroll
+                for (int c = 0; c < 8; ++c) codes[c] &= MAG;
+            }
+            store_words<WPO>(static_cast<char*>(dst) + (e0 + p0) * (F::K / 8), packed);
+
+            // statistics of the row's 8 elements; group sums are flushed where a lane's run crosses a group
+            const uint64_t i0 = first_index + e0 + p0;
+            uint64_t grp = 0, grp_end = ~0ull;
+            double ge = 0.0, ge2 = 0.0;
+            if (group_size) { grp = i0 / group_size; grp_end = (grp + 1) * group_size; }
+            // the row's eight errors first, then their sums as short trees in a fixed order (no long dependent chain)
+            double e[8];
+            uint32_t n_fin = 0, n_up = 0;
+#pragma unroll
+            for (int c = 0; c < 8; ++c) {
+                uint32_t up = 0;
+                e[c] = 0.0;
+                if (stats_element<FMT>(__float_as_uint(y[c]), codes[c], acc, e[c], up)) {
+                    n_fin += 1; n_up += up;
+                    if (group_size) {
+                        while (i0 + c >= grp_end) {
+                            if (ge != 0.0 || ge2 != 0.0) { atomicAdd(gsum_e + grp, ge); atomicAdd(gsum_e2 + grp, ge2); }
+                            ge = 0.0; ge2 = 0.0;
+                            grp = (i0 + c) / group_size; grp_end = (grp + 1) * group_size;
+                        }
+                        ge += e[c]; ge2 = fma(e[c], e[c], ge2);
+                    }
+                }
+            }
+            if (group_size && (ge != 0.0 || ge2 != 0.0)) { atomicAdd(gsum_e + grp, ge); atomicAdd(gsum_e2 + grp, ge2); }
+            acc.n_finite += n_fin; acc.n_up += n_up;
+            double s[8];
+#pragma unroll
+            for (int c = 0; c < 8; ++c) s[c] = (__float_as_uint(y[c]) >> 31) ? -e[c] : e[c];
+            acc.sum_e += ((e[0] + e[1]) + (e[2] + e[3])) + ((e[4] + e[5]) + (e[6] + e[7]));
+            acc.sum_signed_e += ((s[0] + s[1]) + (s[2] + s[3])) + ((s[4] + s[5]) + (s[6] + s[7]));
+            acc.sum_abs_e += ((fabs(e[0]) + fabs(e[1])) + (fabs(e[2]) + fabs(e[3]))) +
+                             ((fabs(e[4]) + fabs(e[5])) + (fabs(e[6]) + fabs(e[7])));
+            acc.sum_e2 += (fma(e[0], e[0], e[1] * e[1]) + fma(e[2], e[2], e[3] * e[3])) +
+                          (fma(e[4], e[4], e[5] * e[5]) + fma(e[6], e[6], e[7] * e[7]));
         }
-        if (group_size && (ge != 0.0 || ge2 != 0.0)) {
-            // the group of the row's last SR-rounded element
-            atomicAdd(gsum_e + grp, ge); atomicAdd(gsum_e2 + grp, ge2);
-        }
-        store_codes8<FMT>(dst, i0, codes);
+        if constexpr (DRAWS && !OWN_CALL) __syncwarp();      // the buffer is rewritten by the next tile
     }
     stats_cta_reduce(acc);
     if (threadIdx.x == 0) partials[blockIdx.x] = acc;
