@@ -329,6 +329,12 @@ int fbsr_round_host(const float* src_host, void* dst_host, size_t n, int fmt, in
     const size_t max_chunk = (size_t)1 << 26;               // keeps the first copy from delaying the first kernel
     if (chunk > max_chunk) chunk = max_chunk / tile * tile;
     if (chunk == 0) return FBSR_ERR_WORKSPACE;
+    // The codes of the last chunk travel back with nothing left to overlap them, so a large call is cut into at
+    // least 8 chunks (of at least 2^21 elements, where a copy is still long against its fixed costs).
+    size_t target = (n + 7) / 8;
+    if (target < ((size_t)1 << 21)) target = (size_t)1 << 21;
+    target = (target + tile - 1) / tile * tile;
+    if (chunk > target) chunk = target;
     // equal chunks (rounded up to whole tiles) instead of full chunks plus a sliver
     const size_t n_chunks = (n + chunk - 1) / chunk;
     chunk = ((n + n_chunks - 1) / n_chunks + tile - 1) / tile * tile;
@@ -350,7 +356,6 @@ int fbsr_round_host(const float* src_host, void* dst_host, size_t n, int fmt, in
         if (cudaMemcpyAsync(slot_in[sl], src_host + at, len * 4, cudaMemcpyHostToDevice, main) != cudaSuccess) return FBSR_ERR_CUDA;
         CallArgs a = base_args(OP_ROUND, variant, k_bits, len, seed, offset + at, slot_out[sl], main);
         a.ovf_ieee = ovf_ieee;
-    a.ovf_ieee = ovf_ieee;
         a.src = reinterpret_cast<const float*>(slot_in[sl]); a.scale = scale;
         if (kRound[fmt](a) != 0) return FBSR_ERR_UNSUPPORTED;
         if (cudaEventRecord(s.rounded[sl], main) != cudaSuccess) return FBSR_ERR_CUDA;
