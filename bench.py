@@ -300,6 +300,21 @@ def main():
                 torch.cuda.synchronize()
                 t8["%s/srf/k%d" % (fmt, k)] = round(5.0 * (1 << 27) / (a.elapsed_time(b) / 10 * 1e-3) / 1e9, 1)
         extras["round_fp8_GBps"] = t8
+        # rounding with the fused error statistics (the call reads the totals back, so each iteration synchronises)
+        ts = {}
+        for fmt, k in (("bf16", 2), ("e4m3", 3)):
+            cb = 2 if fmt == "bf16" else 1
+            outs = torch.empty(1 << 27, dtype=fbsr.CODE_DTYPE[fmt], device=dev)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            fbsr.fbsr_round_stats(x8, fmt, "srf", k, seed=7, scale=2.0 ** -10, out=outs)
+            a.record(stream)
+            for _ in range(5):
+                fbsr.fbsr_round_stats(x8, fmt, "srf", k, seed=7, scale=2.0 ** -10, out=outs)
+            b.record(stream)
+            torch.cuda.synchronize()
+            ts["%s/srf/k%d" % (fmt, k)] = round((4.0 + cb) * (1 << 27) / (a.elapsed_time(b) / 5 * 1e-3) / 1e9, 1)
+            del outs
+        extras["round_stats_GBps"] = ts
         # a format described at run time (general kernel): float8_e4m3fnuz = (8, 4, 8; 240), 5 B/element
         desc = fbsr.format_desc(8, 4, 8, 0x7F, None, 0x80, True)
         td = {}

@@ -8,8 +8,8 @@ import math
 
 import torch
 
-FORMAT_MAX = {"bf16": 3.3895313892515355e38, "fp16": 65504.0, "e4m3": 448.0, "e5m2": 57344.0}
-FORMAT_MIN_NORMAL = {"bf16": 2.0 ** -126, "fp16": 2.0 ** -14, "e4m3": 2.0 ** -6, "e5m2": 2.0 ** -14}
+FORMAT_MAX = {"bf16": 3.3895313892515355e38, "fp16": 65504.0, "e4m3": 448.0, "e5m2": 57344.0, "b8p4": 224.0}
+FORMAT_MIN_NORMAL = {"bf16": 2.0 ** -126, "fp16": 2.0 ** -14, "e4m3": 2.0 ** -6, "e5m2": 2.0 ** -14, "b8p4": 2.0 ** -7}
 
 
 def _gen(seed, device):
@@ -73,7 +73,7 @@ def fp8_activations(fmt, rows=4096, cols=32768, seed=7, device="cpu"):
     x[over] = sgn * (FORMAT_MAX[fmt] / scale) * (1.0 + 15.0 * torch.rand(k, generator=g, device=device))
     sgn = torch.where(torch.rand(k, generator=g, device=device) < 0.5, -1.0, 1.0)
     # magnitudes log-uniform over [2^-(P+5), 1) x min-normal: reaches below half the smallest subnormal
-    span = {"e4m3": 9.0, "e5m2": 8.0, "fp16": 16.0, "bf16": 13.0}[fmt]
+    span = {"e4m3": 9.0, "e5m2": 8.0, "fp16": 16.0, "bf16": 13.0, "b8p4": 9.0}[fmt]
     x[sub] = sgn * (FORMAT_MIN_NORMAL[fmt] / scale) * torch.exp2(-span * torch.rand(k, generator=g, device=device))
     s = min(64, max(n // 64, 1))
     sp = pos[2 * k:2 * k + 3 * s]

@@ -160,7 +160,7 @@ def test_fig1_bias_grid_on_gpu():
             assert np.allclose(ge.cpu().numpy(), ege, rtol=0, atol=1e-9)
 
 
-@pytest.mark.parametrize("fmt", ["e4m3", "e5m2"])
+@pytest.mark.parametrize("fmt", ["e4m3", "e5m2", "b8p4"])
 def test_fp8_activation_workload(fmt):
     """Config 'fp8 path' at 512 x 4096: Laplace activations, amax scaling, saturating outliers,
     subnormal-range values, NaN and +-Inf."""
