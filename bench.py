@@ -292,7 +292,8 @@ def main():
         for fmt in ("e4m3", "e5m2", "b8p4"):
             for k in (2, 4, 8):
                 a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                fbsr.fbsr_round(x8, fmt, "srf", k, seed=7, scale=2.0 ** -10, out=out8)
+                for _ in range(3):
+                    fbsr.fbsr_round(x8, fmt, "srf", k, seed=7, scale=2.0 ** -10, out=out8)
                 a.record(stream)
                 for _ in range(10):
                     fbsr.fbsr_round(x8, fmt, "srf", k, seed=7, scale=2.0 ** -10, out=out8)
