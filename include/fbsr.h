@@ -137,8 +137,9 @@ int fbsr_round_lp(const void* src, int src_fmt, void* dst, size_t n, int dst_fmt
  *                Binary8P4; a zero result then has no sign
  *   ovf_ieee non-zero: finite |y| > M are rounded as IEEE nearest-even does (see FBSR_OVF_IEEE)
  * Special values follow the conventions at the top of this file (Inf -> the infinity, or +-M without one).
- * One general kernel serves every descriptor, any alignment and any offset (vector accesses when src is
- * 16-byte and dst 8 x code-size aligned); it is several times slower than the built-in formats' kernels.
+ * Whole tiles of the draw stream (src 32-byte aligned and dst 8 x code-size aligned at the first tile boundary) are
+ * served by a tiled kernel at roughly half the speed of the built-in formats' kernels; the head, the ragged end and
+ * unaligned calls by a general kernel (any alignment, any offset) that is several times slower.
  * The built-in formats written as descriptors give the built-in results bit for bit.
  * Returns FBSR_ERR_INVALID_ARG for a descriptor outside the ranges above. */
 typedef struct {

@@ -1,7 +1,9 @@
-// fbsr_round_desc: rounding to a format (K, P, B; M) that is described at run time (Section II).
-// One kernel for every such format, with the format's constants as kernel arguments.  A thread takes 8
-// consecutive elements (vector accesses when the pointers allow) and computes the one or two generator
-// calls that cover them from their global indices.
+// fbsr_round_desc: rounding to a format (K, P, B; M) that is described at run time (Section II); the format's
+// constants are kernel arguments.  Two kernels: descriptor_tile_kernel for whole tiles of the draw stream (variant
+// and draw width compile-time, generator calls shared through the warp's buffer), and descriptor_kernel, fully
+// general (run-time variant and draw width, any alignment and offset), for the head, the ragged end and unaligned
+// calls.  In the general kernel a thread takes 8 consecutive elements (vector accesses when the pointers allow) and
+// computes the one or two generator calls that cover them from their global indices.
 // Rounding: as in the tiled kernels, |y| is first multiplied by 2^(1 - EMINB), toward zero, so that the
 // target's exponent range starts where binary32's does; then Eq. (2)-(5) are one addition on the pattern
 // with sh0 = 24 - P excess bits: code = (pattern + (n << (sh0 - N))) >> sh0.  This needs N <= sh0 excess
@@ -10,9 +12,11 @@
 // through the element-wise integer rounder.
 #include <cmath>
 #include <cstring>
+#include <utility>
 
 #include "../../include/fbsr.h"
 #include "fbsr_device.cuh"
+#include "fbsr_kernels.cuh"
 #include "fbsr_internal.h"
 
 namespace fbsr {
@@ -118,6 +122,183 @@ descriptor_kernel(const float* __restrict__ src, void* __restrict__ dst, const u
     }
 }
 
+// Whole tiles with the variant and the draw width fixed at compile time and only the format left to run time:
+// the generator calls of a tile are shared through the warp's buffer and the fields are taken from the packed
+// word stream, as in the bandwidth kernel; a lane owns 8 consecutive elements of a 256-element row.
+// one_addition: the draw fits under the format's 24 - P excess bits (decided by the host, uniform for the launch).
+template <int VAR, int N, int CODE_BYTES>
+__global__ void __launch_bounds__(CTA_THREADS, 4)
+descriptor_tile_kernel(const float* __restrict__ src, const float scale, void* __restrict__ dst, const uint64_t n_tiles,
+                       const uint64_t call0, const uint32_t k0, const uint32_t k1, const RtFormat f,
+                       const bool ieee_overflow, const bool one_addition)
+{
+    using T = Tile<N, 1>;
+    constexpr bool DRAWS = VAR < RTNE;
+    constexpr bool OWN_CALL = T::DPW == 2;
+    constexpr int ROWS = T::ELEMS / ROW_ELEMS;
+    __shared__ __align__(16) uint32_t wordbuf[WARPS_PER_CTA][OWN_CALL ? 4 : T::WORDS + 4];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    uint32_t* wb = wordbuf[warp];
+    const int sh0 = 24 - f.P;
+    const int pos = DRAWS ? sh0 - N : sh0;                   // >= 0 whenever one_addition holds
+    const uint32_t half = pos > 0 ? 1u << (pos - 1) : 0u;
+    const uint32_t below_half = half ? half - 1u : 0u;
+    constexpr bool STICKY = VAR == SRC || VAR == RTNE || VAR == RTO;
+    const float rescale = __uint_as_float((uint32_t)(128 - f.EMINB) << 23);            // 2^(1 - EMINB)
+    const uint32_t max_pattern = f.MAXCODE << sh0;
+    const uint32_t fast_limit = ieee_overflow ? f.MAXBITS : 0x7F7FFFFFu;
+    const uint32_t sign_shift = 32u - (uint32_t)(8 * CODE_BYTES);
+
+    for (uint64_t tile = (uint64_t)blockIdx.x * WARPS_PER_CTA + warp; tile < n_tiles;
+         tile += (uint64_t)gridDim.x * WARPS_PER_CTA) {
+        const size_t e0 = (size_t)tile * T::ELEMS;
+        const uint64_t tile_call0 = call0 + tile * T::CALLS;
+        constexpr int BATCH = ROWS < 4 ? ROWS : (ROWS % 3 == 0 ? 3 : (ROWS % 2 == 0 ? 2 : ROWS));
+        F8 regs[BATCH];
+#pragma unroll
+        for (int j = 0; j < BATCH; ++j) regs[j] = load_f8_stream(src + e0 + j * ROW_ELEMS + lane * 8);
+        if constexpr (DRAWS && !OWN_CALL) {
+#pragma unroll
+            for (int j = 0; j < (T::CALLS + 31) / 32; ++j) {
+                const int c = j * 32 + lane;
+                if (T::CALLS % 32 == 0 || c < T::CALLS)
+                    *reinterpret_cast<uint4*>(wb + 4 * c) = philox_block(tile_call0 + c, k0, k1);
+            }
+            __syncwarp();
+        }
+#pragma unroll
+        for (int rb = 0; rb < ROWS; rb += BATCH) {
+            if (rb > 0) {
+#pragma unroll
+                for (int j = 0; j < BATCH; ++j)
+                    if (rb + j < ROWS) regs[j] = load_f8_stream(src + e0 + (rb + j) * ROW_ELEMS + lane * 8);
+            }
+#pragma unroll
+            for (int j = 0; j < BATCH; ++j) {
+                if (rb + j >= ROWS) continue;
+                const int p0 = (rb + j) * ROW_ELEMS + lane * 8;
+                float x[8];
+                unpack(regs[j], x);
+                Draws8<N> d;
+                if constexpr (!DRAWS) {
+                } else if constexpr (OWN_CALL) {
+                    d.from_call(philox_block(tile_call0 + p0 / 8, k0, k1));
+                } else {
+                    d.from_stream(wb, p0);
+                }
+                uint32_t codes[8];
+#pragma unroll
+                for (int c = 0; c < 8; ++c) {
+                    const uint32_t yb = scaled_bits(x[c], scale);
+                    const uint32_t mbits = yb & 0x7FFFFFFFu;
+                    const uint32_t nr = DRAWS ? d.template at<0>(c) : 0u;
+                    if (one_addition && mbits <= fast_limit) {
+                        const float mag = __uint_as_float(mbits);
+                        uint32_t u = __float_as_uint(__fmul_rz(mag, rescale));
+                        if constexpr (STICKY) u |= (u ^ __float_as_uint(__fmul_ru(mag, rescale))) & 1u;
+                        u = min(u, max_pattern);
+                        uint32_t sum;
+                        if constexpr (VAR == SRFF) sum = u + (nr << pos);
+                        else if constexpr (VAR == SRF) sum = u + half + (nr << pos);
+                        else if constexpr (VAR == RTA) sum = u + half;
+                        else sum = u + below_half + (((u >> pos) & 1u) ^ (VAR == RTO ? 1u : 0u)) + (DRAWS ? nr << pos : 0u);
+                        const uint32_t code = sum >> sh0;
+                        codes[c] = (f.SINGLE_ZERO && code == 0u) ? 0u : (code | ((yb >> 31) << (31u - sign_shift)));
+                    } else {
+                        codes[c] = round_core_fmt<RtFormat, false, false>(f, yb, nr, VAR, N, nullptr, ieee_overflow);
+                    }
+                }
+                if constexpr (CODE_BYTES == 2) {
+                    const uint32_t w[4] = {codes[0] | (codes[1] << 16), codes[2] | (codes[3] << 16),
+                                           codes[4] | (codes[5] << 16), codes[6] | (codes[7] << 16)};
+                    store_words<4>(static_cast<char*>(dst) + (e0 + p0) * 2, w);
+                } else {
+                    const uint32_t w[2] = {codes[0] | (codes[1] << 8) | (codes[2] << 16) | (codes[3] << 24),
+                                           codes[4] | (codes[5] << 8) | (codes[6] << 16) | (codes[7] << 24)};
+                    store_words<2>(static_cast<char*>(dst) + (e0 + p0), w);
+                }
+            }
+        }
+        if constexpr (DRAWS && !OWN_CALL) __syncwarp();      // the buffer is rewritten by the next tile
+    }
+}
+
+struct TileCall {
+    const float* src; void* dst; uint64_t n_tiles, call0; float scale; uint32_t k0, k1; RtFormat f;
+    bool ieee_overflow, one_addition; cudaStream_t stream;
+};
+
+template <int VAR, int N>
+void launch_descriptor_tiles(const TileCall& t)
+{
+    const uint64_t want = (t.n_tiles + WARPS_PER_CTA - 1) / WARPS_PER_CTA;
+    const unsigned grid = (unsigned)(want < 0x7FFFFFF0ull ? want : 0x7FFFFFF0ull);
+    if (t.f.K == 16) {
+        descriptor_tile_kernel<VAR, N, 2><<<grid, CTA_THREADS, 0, t.stream>>>(t.src, t.scale, t.dst, t.n_tiles, t.call0, t.k0,
+                                                                            t.k1, t.f, t.ieee_overflow, t.one_addition);
+    } else {
+        descriptor_tile_kernel<VAR, N, 1><<<grid, CTA_THREADS, 0, t.stream>>>(t.src, t.scale, t.dst, t.n_tiles, t.call0, t.k0,
+                                                                            t.k1, t.f, t.ieee_overflow, t.one_addition);
+    }
+    count_launch();
+}
+
+template <int VAR>
+void descriptor_tiles_by_k(int k, const TileCall& t)
+{
+    switch (k) {
+    case 1: return launch_descriptor_tiles<VAR, 1>(t);
+    case 2: return launch_descriptor_tiles<VAR, 2>(t);
+    case 3: return launch_descriptor_tiles<VAR, 3>(t);
+    case 4: return launch_descriptor_tiles<VAR, 4>(t);
+    case 5: return launch_descriptor_tiles<VAR, 5>(t);
+    case 6: return launch_descriptor_tiles<VAR, 6>(t);
+    case 7: return launch_descriptor_tiles<VAR, 7>(t);
+    case 8: return launch_descriptor_tiles<VAR, 8>(t);
+    case 9: return launch_descriptor_tiles<VAR, 9>(t);
+    case 10: return launch_descriptor_tiles<VAR, 10>(t);
+    case 11: return launch_descriptor_tiles<VAR, 11>(t);
+    case 12: return launch_descriptor_tiles<VAR, 12>(t);
+    case 13: return launch_descriptor_tiles<VAR, 13>(t);
+    case 14: return launch_descriptor_tiles<VAR, 14>(t);
+    case 15: return launch_descriptor_tiles<VAR, 15>(t);
+    default: return launch_descriptor_tiles<VAR, 16>(t);
+    }
+}
+
+// Elements per tile for k bits per draw (the deterministic modes use the 1024-element tile of k = 16).
+template <int... Ks>
+size_t tile_elements_of(int k, std::integer_sequence<int, Ks...>)
+{
+    static constexpr size_t table[16] = {(size_t)Tile<Ks + 1, 1>::ELEMS...};
+    return table[k - 1];
+}
+size_t descriptor_tile_elements(int variant, int k)
+{
+    return tile_elements_of(variant >= RTNE ? 16 : k, std::make_integer_sequence<int, 16>{});
+}
+
+// The general kernel on elements [begin, end) of the call.
+void launch_descriptor_general(const float* src, void* dst, size_t begin, size_t end, const RtFormat& f, int variant, int k,
+                               uint64_t seed, uint64_t offset, float scale, bool ieee, cudaStream_t stream)
+{
+    if (begin >= end) return;
+    const size_t n = end - begin, cb = (size_t)f.K / 8;
+    const float* s = src + begin;
+    void* d = static_cast<char*>(dst) + begin * cb;
+    const bool vectors = reinterpret_cast<uintptr_t>(s) % 16 == 0 && reinterpret_cast<uintptr_t>(d) % (8 * cb) == 0;
+    const uint64_t n_octets = ((uint64_t)n + 7) / 8;
+    const uint64_t want = (n_octets + DESC_THREADS - 1) / DESC_THREADS;
+    const unsigned grid = (unsigned)(want < 0x7FFFFFF0ull ? want : 0x7FFFFFF0ull);
+    const uint32_t E = 4u * (32u / (uint32_t)k);
+    const uint64_t g0 = offset + begin;
+    const uint32_t first_field = (uint32_t)(g0 % E);
+    const bool short_call = (uint64_t)n + first_field + 8u < 0xFFFFFFFFull;
+    descriptor_kernel<<<grid, DESC_THREADS, 0, stream>>>(s, d, (uint64_t)n, g0 / E, first_field, short_call, scale, f, variant, k,
+                                                         (uint32_t)seed, (uint32_t)(seed >> 32), ieee, vectors);
+    count_launch();
+}
+
 // Checks the descriptor and fills in the constants the rounder needs.  Returns false if it is not accepted.
 bool make_rt_format(const fbsr_format_desc* d, RtFormat* f)
 {
@@ -169,16 +350,34 @@ extern "C" int fbsr_round_desc(const float* src, void* dst, size_t n, const fbsr
     const size_t code_bytes = (size_t)f.K / 8;
     if (reinterpret_cast<uintptr_t>(src) % 4 != 0 || reinterpret_cast<uintptr_t>(dst) % code_bytes != 0) return FBSR_ERR_ALIGNMENT;
     if (n == 0) return FBSR_OK;
-    const bool vectors = reinterpret_cast<uintptr_t>(src) % 16 == 0 && reinterpret_cast<uintptr_t>(dst) % (8 * code_bytes) == 0;
-    const uint64_t n_octets = ((uint64_t)n + 7) / 8;
-    const uint64_t want = (n_octets + DESC_THREADS - 1) / DESC_THREADS;
-    const unsigned grid = (unsigned)(want < 0x7FFFFFF0ull ? want : 0x7FFFFFF0ull);
-    const uint32_t E = 4u * (32u / (uint32_t)k_bits);
-    const uint32_t first_field = (uint32_t)(offset % E);
-    const bool short_call = (uint64_t)n + first_field + 8u < 0xFFFFFFFFull;
-    descriptor_kernel<<<grid, DESC_THREADS, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
-        src, dst, (uint64_t)n, offset / E, first_field, short_call, scale, f, variant, k_bits, (uint32_t)seed, (uint32_t)(seed >> 32),
-        ovf_ieee != 0, vectors);
-    count_launch();
+    const cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const bool ieee = ovf_ieee != 0;
+    // Whole tiles of the draw stream go to the tiled kernel when the pointers allow its vector accesses; the head
+    // before the first tile boundary, the ragged end, and calls with unaligned pointers go to the general kernel.
+    const size_t tile = descriptor_tile_elements(variant, k_bits);
+    const size_t head = (size_t)((tile - offset % tile) % tile);
+    size_t n_tiles = 0;
+    if (head < n && reinterpret_cast<uintptr_t>(src + head) % 32 == 0 &&
+        reinterpret_cast<uintptr_t>(static_cast<char*>(dst) + head * code_bytes) % (8 * code_bytes) == 0)
+        n_tiles = (n - head) / tile;
+    if (n_tiles == 0) {
+        launch_descriptor_general(src, dst, 0, n, f, variant, k_bits, seed, offset, scale, ieee, stream);
+    } else {
+        const int needed = variant == SRF ? k_bits + 1 : variant == SRC ? k_bits + 2 : k_bits;
+        const int k_tile = variant >= RTNE ? 16 : k_bits;
+        TileCall t{src + head, static_cast<char*>(dst) + head * code_bytes, n_tiles,
+                   (offset + head) / (4u * (32u / (uint32_t)k_tile)), scale, (uint32_t)seed, (uint32_t)(seed >> 32), f, ieee,
+                   variant >= RTNE || needed <= 24 - f.P, stream};
+        launch_descriptor_general(src, dst, 0, head, f, variant, k_bits, seed, offset, scale, ieee, stream);
+        switch (variant) {
+        case SRFF: descriptor_tiles_by_k<SRFF>(k_bits, t); break;
+        case SRF: descriptor_tiles_by_k<SRF>(k_bits, t); break;
+        case SRC: descriptor_tiles_by_k<SRC>(k_bits, t); break;
+        case RTNE: launch_descriptor_tiles<RTNE, 16>(t); break;
+        case RTA: launch_descriptor_tiles<RTA, 16>(t); break;
+        default: launch_descriptor_tiles<RTO, 16>(t); break;
+        }
+        launch_descriptor_general(src, dst, head + n_tiles * tile, n, f, variant, k_bits, seed, offset, scale, ieee, stream);
+    }
     return cudaGetLastError() == cudaSuccess ? FBSR_OK : FBSR_ERR_CUDA;
 }
