@@ -136,7 +136,7 @@ descriptor_tile_kernel(const float* __restrict__ src, const float scale, void* _
     constexpr bool DRAWS = VAR < RTNE;
     constexpr bool OWN_CALL = T::DPW == 2;
     constexpr int ROWS = T::ELEMS / ROW_ELEMS;
-    __shared__ __align__(16) uint32_t wordbuf[WARPS_PER_CTA][OWN_CALL ? 4 : T::WORDS + 4];
+    __shared__ __align__(16) uint32_t wordbuf[WARPS_PER_CTA][OWN_CALL ? 4 : T::BUFFER_WORDS];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     uint32_t* wb = wordbuf[warp];
     const int sh0 = 24 - f.P;
@@ -162,7 +162,7 @@ descriptor_tile_kernel(const float* __restrict__ src, const float scale, void* _
             for (int j = 0; j < (T::CALLS + 31) / 32; ++j) {
                 const int c = j * 32 + lane;
                 if (T::CALLS % 32 == 0 || c < T::CALLS)
-                    *reinterpret_cast<uint4*>(wb + 4 * c) = philox_block(tile_call0 + c, k0, k1);
+                    Draws8<N>::store_call(wb + Draws8<N>::WORDS_PER_CALL * c, philox_block(tile_call0 + c, k0, k1));
             }
             __syncwarp();
         }
@@ -184,7 +184,7 @@ descriptor_tile_kernel(const float* __restrict__ src, const float scale, void* _
                 } else if constexpr (OWN_CALL) {
                     d.from_call(philox_block(tile_call0 + p0 / 8, k0, k1));
                 } else {
-                    d.from_stream(wb, p0);
+                    d.from_normalised(wb, p0);
                 }
                 uint32_t codes[8];
 #pragma unroll

@@ -260,6 +260,46 @@ template <int K> struct Draws8 {
         }
     }
 
+    // Normalised layout (used where the generator fills the buffer): for draw counts per word that are not a power
+    // of two the lane that computes a call writes its E fields as E / G words of G fields each, so that an octet of
+    // elements later reads 8 / G ready words instead of joining raw words itself.  Power-of-two counts keep the raw
+    // layout, which is already normalised.
+    static constexpr int E = 4 * DPW;
+    static constexpr int WORDS_PER_CALL = POW2 ? 4 : E / G;
+    static_assert(POW2 || E % G == 0, "a call splits into whole groups");
+
+    __device__ __forceinline__ static void store_call(uint32_t* dst, const uint4& o)
+    {
+        if constexpr (POW2) {
+            *reinterpret_cast<uint4*>(dst) = o;
+        } else {
+            // the call's fields as one bit sequence: each word contributes its low DPW * K bits
+            constexpr int B = DPW * K;
+            constexpr uint32_t PAYLOAD = (uint32_t)((1ull << B) - 1ull);
+            const unsigned __int128 seq = (unsigned __int128)(o.x & PAYLOAD) | ((unsigned __int128)(o.y & PAYLOAD) << B) |
+                                          ((unsigned __int128)(o.z & PAYLOAD) << (2 * B)) |
+                                          ((unsigned __int128)(o.w & PAYLOAD) << (3 * B));
+#pragma unroll
+            for (int m = 0; m < WORDS_PER_CALL; ++m) dst[m] = (uint32_t)(seq >> (m * G * K));
+        }
+    }
+
+    // From the tile's buffer in the normalised layout; p0 = tile-relative index of the lane's first element.
+    __device__ __forceinline__ void from_normalised(const uint32_t* wb, const int p0)
+    {
+        if constexpr (POW2) {
+            from_stream(wb, p0);
+        } else if constexpr (G == 8) {
+            u[0] = wb[p0 / 8];
+        } else if constexpr (G == 4) {
+            const uint2 w = *reinterpret_cast<const uint2*>(wb + p0 / 4);
+            u[0] = w.x; u[1] = w.y;
+        } else {
+            const uint4 w = *reinterpret_cast<const uint4*>(wb + p0 / 2);
+            u[0] = w.x; u[1] = w.y; u[2] = w.z; u[3] = w.w;
+        }
+    }
+
     // From one Philox call that serves exactly these 8 elements (two draws per word).
     __device__ __forceinline__ void from_call(const uint4& w)
     {

@@ -67,6 +67,7 @@ template <int K, int OCT = 1> struct Tile {
     static constexpr int ELEMS = ROWS1 * ROW_ELEMS * (ROWS1 % OCT == 0 ? 1 : 2);
     static constexpr int CALLS = ELEMS / E;                   // Philox calls per tile
     static constexpr int WORDS = ELEMS / DPW;                 // random words per tile
+    static constexpr int BUFFER_WORDS = CALLS * Draws8<K>::WORDS_PER_CALL;   // of the generator-filled buffer
     static constexpr uint32_t MASK = (1u << K) - 1u;
     static_assert(ELEMS % E == 0, "a tile must hold whole Philox calls");
 };
@@ -647,7 +648,9 @@ tile_kernel(const Op op, void* __restrict__ dst, const uint64_t n_tiles, const u
         return;
     }
     constexpr bool OWN_CALL = (T::DPW == 2) && !BITS;      // a call serves exactly one lane-row
-    __shared__ __align__(16) uint32_t wordbuf[WARPS_PER_CTA][OWN_CALL ? 4 : T::WORDS + 4];   // +4: the joined-word read of the last group
+    // supplied words keep their packed layout (+4: the joined-word read of the last group); generated ones are
+    // written in the normalised layout of Draws8
+    __shared__ __align__(16) uint32_t wordbuf[WARPS_PER_CTA][OWN_CALL ? 4 : (BITS ? T::WORDS + 4 : T::BUFFER_WORDS)];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     uint32_t* wb = wordbuf[warp];
 
@@ -681,7 +684,7 @@ tile_kernel(const Op op, void* __restrict__ dst, const uint64_t n_tiles, const u
             for (int j = 0; j < (T::CALLS + 31) / 32; ++j) {
                 const int c = j * 32 + lane;
                 if (T::CALLS % 32 == 0 || c < T::CALLS)
-                    *reinterpret_cast<uint4*>(wb + 4 * c) = philox_block(tile_call0 + c, k0, k1);
+                    Draws8<K>::store_call(wb + Draws8<K>::WORDS_PER_CALL * c, philox_block(tile_call0 + c, k0, k1));
             }
             __syncwarp();
         }
@@ -708,8 +711,10 @@ tile_kernel(const Op op, void* __restrict__ dst, const uint64_t n_tiles, const u
                         if constexpr (!DRAWS) {
                         } else if constexpr (OWN_CALL) {
                             d.from_call(philox_block(tile_call0 + po / 8, k0, k1));
-                        } else {
+                        } else if constexpr (BITS) {
                             d.from_stream(wb, po);
+                        } else {
+                            d.from_normalised(wb, po);
                         }
                         uint32_t t[8];
                         const bool redo = round_row_fast<FMT, VAR, K>(y, d, t);
@@ -911,7 +916,7 @@ stats_tile_kernel(const float* __restrict__ src, const float scale, void* __rest
     constexpr int ROWS = T::ELEMS / ROW_ELEMS;
     constexpr int WPO = WordsPerOctet<FMT>::value;
     constexpr uint32_t MAG = (1u << (F::K - 1)) - 1u;
-    __shared__ __align__(16) uint32_t wordbuf[WARPS_PER_CTA][OWN_CALL ? 4 : T::WORDS + 4];
+    __shared__ __align__(16) uint32_t wordbuf[WARPS_PER_CTA][OWN_CALL ? 4 : T::BUFFER_WORDS];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     uint32_t* wb = wordbuf[warp];
     StatsAcc acc;
@@ -931,7 +936,7 @@ stats_tile_kernel(const float* __restrict__ src, const float scale, void* __rest
             for (int j = 0; j < (T::CALLS + 31) / 32; ++j) {
                 const int c = j * 32 + lane;
                 if (T::CALLS % 32 == 0 || c < T::CALLS)
-                    *reinterpret_cast<uint4*>(wb + 4 * c) = philox_block(tile_call0 + c, k0, k1);
+                    Draws8<K>::store_call(wb + Draws8<K>::WORDS_PER_CALL * c, philox_block(tile_call0 + c, k0, k1));
             }
             __syncwarp();
         }
@@ -948,7 +953,7 @@ stats_tile_kernel(const float* __restrict__ src, const float scale, void* __rest
             } else if constexpr (OWN_CALL) {
                 d.from_call(philox_block(tile_call0 + p0 / 8, k0, k1));
             } else {
-                d.from_stream(wb, p0);
+                d.from_normalised(wb, p0);
             }
             uint32_t t[8], codes[8], packed[WPO];
             const bool redo = round_row_fast<FMT, VAR, K>(y, d, t);
