@@ -42,8 +42,8 @@ def sweep():
 # DRAM traffic of one 2^28-element bf16 launch, from the ncu capture summarised in
 # profiles/tile_kernel_round.txt (dram__bytes_read.sum + dram__bytes_write.sum of a 2^27-element
 # launch, scaled by the elements processed).  Valid only for the kernel sources it was taken from.
-TRAFFIC_BYTES_PER_LAUNCH = 2 * (536.965632e6 + 221.757696e6)
-TRAFFIC_KERNEL_SHA = "64b0f4076d9edb9f"
+TRAFFIC_BYTES_PER_LAUNCH = 2 * (536.893952e6 + 221.408768e6)
+TRAFFIC_KERNEL_SHA = "358d6c0691e7a25d"
 
 
 def kernel_source_sha():
