@@ -73,8 +73,7 @@ typedef enum {
 /* May be or-ed into any `fmt` argument.  Section II says that values beyond the finite range are "rounded
  * deterministically as in IEEE-754 round to nearest"; with this flag finite |y| > M follow that reading
  * (M below M + ulp(M)/2, +-Inf above it -- the NaN code for e4m3 -- ties to the even neighbour) instead
- * of saturating.  Rows of 8 elements that hold such a value are rounded element by element; the others run
- * at full speed (fbsr_round_stats with the flag runs on the general, slower kernel). */
+ * of saturating.  Calls with the flag run on the general (slower) kernel. */
 #define FBSR_OVF_IEEE 0x100
 
 /* Round-up predicates: the few-bit stochastic ones of Section II-B and Eq. (8), and the deterministic

@@ -85,7 +85,7 @@ int launch_tiles(const Op& op, const CallArgs& a, const Plan& p)
     const uint64_t call0 = BITS ? 0 : (a.offset + p.head) / T::E;
     const uint32_t* words = BITS ? a.words + p.head / T::DPW : nullptr;
     kern<<<grid, CTA_THREADS, 0, a.stream>>>(adv, dst, p.n_tiles, call0, (uint32_t)a.seed,
-                                             (uint32_t)(a.seed >> 32), words, tail_count, a.ovf_ieee != 0);
+                                             (uint32_t)(a.seed >> 32), words, tail_count);
     count_launch();
     return 0;
 }
@@ -133,7 +133,8 @@ template <class Op, int VAR, int K, bool BITS>
 int run(const Op& op, const CallArgs& a)
 {
     const Plan p = make_plan<Op, K, BITS>(op, a);
-    if (p.n_tiles == 0) return launch_generic<Op, BITS, false>(op, a, 0, a.n, nullptr);
+    // the IEEE-overflow option is served by the general kernel only
+    if (p.n_tiles == 0 || a.ovf_ieee) return launch_generic<Op, BITS, false>(op, a, 0, a.n, nullptr);
     launch_generic<Op, BITS, false>(op, a, 0, p.head, nullptr);
     launch_tiles<Op, VAR, K, BITS>(op, a, p);          // whole tiles and the ragged end
     return 0;

@@ -621,8 +621,7 @@ __device__ __forceinline__ void pack_row_fast(const uint32_t (&t)[8], const floa
 template <class Op, int FMT, int VAR, int K, bool BITS>
 __global__ void __launch_bounds__(CTA_THREADS, Op::MIN_CTAS)
 tile_kernel(const Op op, void* __restrict__ dst, const uint64_t n_tiles, const uint64_t call0,
-            const uint32_t k0, const uint32_t k1, const uint32_t* __restrict__ words, const uint32_t tail_count,
-            const bool ieee_overflow)
+            const uint32_t k0, const uint32_t k1, const uint32_t* __restrict__ words, const uint32_t tail_count)
 {
     using T = Tile<K, Op::OCTETS>;
     constexpr bool DRAWS = VAR < RTNE;                     // the deterministic modes use no random bits
@@ -644,7 +643,7 @@ tile_kernel(const Op op, void* __restrict__ dst, const uint64_t n_tiles, const u
                 word = ws == 0 ? o.x : ws == 1 ? o.y : ws == 2 ? o.z : o.w;
             }
             const uint32_t n = (word >> ((j % T::DPW) * K)) & T::MASK;
-            store_code1<FMT>(dst, p, round_core<FMT, false>(op.scalar(p), n, VAR, K, nullptr, ieee_overflow));
+            store_code1<FMT>(dst, p, round_core<FMT, false>(op.scalar(p), n, VAR, K, nullptr));
         }
         return;
     }
@@ -718,14 +717,7 @@ tile_kernel(const Op op, void* __restrict__ dst, const uint64_t n_tiles, const u
                             d.from_normalised(wb, po);
                         }
                         uint32_t t[8];
-                        bool redo = round_row_fast<FMT, VAR, K>(y, d, t);
-                        if (ieee_overflow) {
-                            // the fast rows saturate; with the IEEE reading of overflow a row holding a finite
-                            // value beyond M is redone element by element as well
-                            const float m_f = __uint_as_float(Format<FMT>::MAXBITS);
-#pragma unroll
-                            for (int i = 0; i < 8; ++i) redo = redo || fabsf(y[i]) > m_f;
-                        }
+                        const bool redo = round_row_fast<FMT, VAR, K>(y, d, t);
                         if (!redo) {
                             pack_row_fast<FMT>(t, y, packed + o * WPO);
                         } else {
@@ -736,7 +728,7 @@ tile_kernel(const Op op, void* __restrict__ dst, const uint64_t n_tiles, const u
                                 uint32_t bits;
                                 if constexpr (OCT == 1) bits = op.exact_bits(regs[j], i, y[i]);
                                 else bits = op.exact_bits(regs[j], o, i, y[i]);
-                                c[i] = round_core<FMT, false>(bits, d.template at<0>(i), VAR, K, nullptr, ieee_overflow);
+                                c[i] = round_core<FMT, false>(bits, d.template at<0>(i), VAR, K, nullptr);
                             }
                             pack_codes8<FMT>(c, packed + o * WPO);
                         }
