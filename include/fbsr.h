@@ -73,7 +73,8 @@ typedef enum {
 /* May be or-ed into any `fmt` argument.  Section II says that values beyond the finite range are "rounded
  * deterministically as in IEEE-754 round to nearest"; with this flag finite |y| > M follow that reading
  * (M below M + ulp(M)/2, +-Inf above it -- the NaN code for e4m3 -- ties to the even neighbour) instead
- * of saturating.  Calls with the flag run on the general (slower) kernel. */
+ * of saturating.  fbsr_round, fbsr_round_bits and fbsr_round_lp serve the flag with a second pass over the input
+ * that rewrites the values beyond M (about a third of the usual speed); the other calls use the general kernel. */
 #define FBSR_OVF_IEEE 0x100
 
 /* Round-up predicates: the few-bit stochastic ones of Section II-B and Eq. (8), and the deterministic

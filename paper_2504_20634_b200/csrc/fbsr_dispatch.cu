@@ -129,14 +129,54 @@ Plan make_plan(const Op& op, const CallArgs& a)
     return p;
 }
 
+// The IEEE reading of overflow after a saturating pass: only finite values beyond M differ (M + ulp/2 and above
+// become the infinity, or the NaN of a format without one), and they need no draw.  For ops whose value can be
+// formed again from their inputs (plain rounding and 16-bit sources) the call runs the tiled kernels as usual and
+// this kernel then rewrites those elements, one element per thread; the other ops use the general kernel.
+template <class Op> struct Restartable { static constexpr bool value = false; };
+template <> struct Restartable<RoundOp> { static constexpr bool value = true; };
+template <int SRC> struct Restartable<LpSrcOp<SRC>> { static constexpr bool value = true; };
+
+template <class Op>
+__global__ void __launch_bounds__(CTA_THREADS)
+overflow_fixup_kernel(const Op op, void* __restrict__ dst, const uint64_t n)
+{
+    // a CTA takes chunks of 8 x 256 elements; a thread's 8 loads are independent and coalesced across the warp
+    constexpr int PER_THREAD = 8;
+    constexpr uint64_t CHUNK = (uint64_t)PER_THREAD * CTA_THREADS;
+    for (uint64_t base = (uint64_t)blockIdx.x * CHUNK; base < n; base += (uint64_t)gridDim.x * CHUNK) {
+        uint32_t bits[PER_THREAD];
+#pragma unroll
+        for (int j = 0; j < PER_THREAD; ++j) {
+            const uint64_t i = base + (uint64_t)j * CTA_THREADS + threadIdx.x;
+            bits[j] = i < n ? op.scalar(i) : 0u;
+        }
+#pragma unroll
+        for (int j = 0; j < PER_THREAD; ++j) {
+            const uint64_t i = base + (uint64_t)j * CTA_THREADS + threadIdx.x;
+            const uint32_t mag = bits[j] & 0x7FFFFFFFu;
+            if (mag > Format<FMT>::MAXBITS && mag < 0x7F800000u)
+                store_code1<FMT>(dst, i, round_core<FMT, false>(bits[j], 0u, RTNE, 1, nullptr, true));
+        }
+    }
+}
+
 template <class Op, int VAR, int K, bool BITS>
 int run(const Op& op, const CallArgs& a)
 {
     const Plan p = make_plan<Op, K, BITS>(op, a);
-    // the IEEE-overflow option is served by the general kernel only
-    if (p.n_tiles == 0 || a.ovf_ieee) return launch_generic<Op, BITS, false>(op, a, 0, a.n, nullptr);
-    launch_generic<Op, BITS, false>(op, a, 0, p.head, nullptr);
+    const bool fixup = a.ovf_ieee && Restartable<Op>::value;
+    if (p.n_tiles == 0 || (a.ovf_ieee && !fixup)) return launch_generic<Op, BITS, false>(op, a, 0, a.n, nullptr);
+    CallArgs sat = a;
+    sat.ovf_ieee = 0;                                  // the head, too, saturates first when the fix-up pass follows
+    launch_generic<Op, BITS, false>(op, sat, 0, p.head, nullptr);
     launch_tiles<Op, VAR, K, BITS>(op, a, p);          // whole tiles and the ragged end
+    if (fixup) {
+        const uint64_t want = ((uint64_t)a.n + 8 * CTA_THREADS - 1) / (8 * CTA_THREADS);
+        const unsigned grid = (unsigned)(want < 0x7FFFFFF0ull ? want : 0x7FFFFFF0ull);
+        overflow_fixup_kernel<Op><<<grid, CTA_THREADS, 0, a.stream>>>(op, a.dst, (uint64_t)a.n);
+        count_launch();
+    }
     return 0;
 }
 
