@@ -173,7 +173,7 @@ int run(const Op& op, const CallArgs& a)
     launch_tiles<Op, VAR, K, BITS>(op, a, p);          // whole tiles and the ragged end
     if (fixup) {
         const uint64_t want = ((uint64_t)a.n + 8 * CTA_THREADS - 1) / (8 * CTA_THREADS);
-        const unsigned grid = (unsigned)(want < 0x7FFFFFF0ull ? want : 0x7FFFFFF0ull);
+        const unsigned grid = (unsigned)(want < (uint64_t)MAX_SLOW_GRID ? want : (uint64_t)MAX_SLOW_GRID);   // resident CTAs loop over the chunks
         overflow_fixup_kernel<Op><<<grid, CTA_THREADS, 0, a.stream>>>(op, a.dst, (uint64_t)a.n);
         count_launch();
     }
