@@ -128,3 +128,24 @@ def test_ieee_overflow_option(fmt):
     mask = 0x7FFF if got.dtype == torch.uint16 else 0x7F
     ok = torch.isfinite(xd)
     assert torch.equal(got.view(as_int)[ok] & mask, ref[ok] & mask)
+
+
+def test_ieee_overflow_option_with_supplied_bits_and_16_bit_sources():
+    """The same option through fbsr_round_bits and fbsr_round_lp (tiled pass, then the pass that rewrites values beyond M)."""
+    rng = np.random.default_rng(99)
+    n = 9 * 1280 + 301
+    x = (np.float32(448.0) * (1.0 + rng.uniform(-0.3, 0.3, n))).astype(np.float32) * np.where(rng.integers(0, 2, n), 1, -1).astype(np.float32)
+    x[:200] = gu.mixed_inputs(200, 6, "e4m3")
+    xd = torch.from_numpy(x).cuda()
+    for fmt in ("e4m3", "e5m2", "b8p4"):
+        for variant, k in (("srf", 3), ("src", 4)):
+            words = capi.random_words(seed=3, offset=0, count=n, k=k)
+            got = fbsr.fbsr_round_bits(xd, fmt + "+ieee", variant, k, gu.from_np_u32(words), scale=0.6)
+            gu.assert_codes_equal(got, capi.fbsr_round_bits(x, fmt + "+ieee", variant, k, words, scale=0.6), "bits " + fmt)
+    codes16 = rng.integers(0, 1 << 16, size=n).astype(np.uint16)          # every kind of bf16 / fp16 code, huge ones included
+    cd = gu.from_np_codes(codes16)
+    for src_fmt in ("bf16", "fp16"):
+        for fmt in ("e4m3", "e5m2", "b8p4"):
+            got = fbsr.fbsr_round_lp(cd, src_fmt, fmt + "+ieee", "src", 3, seed=8, offset=2560, scale=1.5)
+            gu.assert_codes_equal(got, capi.fbsr_round_lp(codes16, src_fmt, fmt + "+ieee", "src", 3, seed=8, offset=2560, scale=1.5),
+                                  "lp %s->%s" % (src_fmt, fmt))
