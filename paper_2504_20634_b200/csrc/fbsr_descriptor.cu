@@ -189,7 +189,7 @@ descriptor_tile_kernel(const float* __restrict__ src, const float scale, void* _
                 uint32_t codes[8];
 #pragma unroll
                 for (int c = 0; c < 8; ++c) {
-                    const uint32_t yb = scaled_bits(x[c], scale);
+                    const uint32_t yb = __float_as_uint(__fmul_rn(x[c], scale));    // a NaN takes the other branch
                     const uint32_t mbits = yb & 0x7FFFFFFFu;
                     const uint32_t nr = DRAWS ? d.template at<0>(c) : 0u;
                     if (one_addition && mbits <= fast_limit) {
@@ -205,7 +205,9 @@ descriptor_tile_kernel(const float* __restrict__ src, const float scale, void* _
                         const uint32_t code = sum >> sh0;
                         codes[c] = (f.SINGLE_ZERO && code == 0u) ? 0u : (code | ((yb >> 31) << (31u - sign_shift)));
                     } else {
-                        codes[c] = round_core_fmt<RtFormat, false, false>(f, yb, nr, VAR, N, nullptr, ieee_overflow);
+                        // scaled_bits: a NaN input keeps its own sign
+                        codes[c] = round_core_fmt<RtFormat, false, false>(f, scaled_bits(x[c], scale), nr, VAR, N, nullptr,
+                                                                          ieee_overflow);
                     }
                 }
                 if constexpr (CODE_BYTES == 2) {
