@@ -217,23 +217,30 @@ def fbsr_round_bits(src, fmt, variant, k_bits, rand_words, scale=1.0, out=None):
 
 
 def fbsr_round_stats(src, fmt, variant, k_bits, seed, offset=0, scale=1.0, group_size=0, out=None,
-                     workspace=None):
+                     workspace=None, total=None, read_back=True):
     """Returns (codes, stats dict, group_sum_e, group_sum_e2); the stats dict is read back with one
-    device-to-host copy after the call."""
+    device-to-host copy after the call.  With read_back=False nothing is copied or synchronised and the
+    second item is the 72-byte device tensor holding the fbsr_stats record (decode it with
+    stats_from_bytes once the stream has been synchronised); `total` and `workspace` may be supplied so
+    that repeated calls allocate nothing."""
     out, po = _out(src, fmt, out)
     n = src.numel()
     groups = (n + group_size - 1) // group_size if group_size else 0
-    ge = torch.empty(max(groups, 1), dtype=torch.float64, device=src.device)
-    ge2 = torch.empty(max(groups, 1), dtype=torch.float64, device=src.device)
-    total = torch.empty(ctypes.sizeof(FbsrStats), dtype=torch.uint8, device=src.device)
+    ge = torch.empty(max(groups, 1), dtype=torch.float64, device=src.device) if groups or read_back else None
+    ge2 = torch.empty(max(groups, 1), dtype=torch.float64, device=src.device) if groups or read_back else None
+    if total is None:
+        total = torch.empty(ctypes.sizeof(FbsrStats), dtype=torch.uint8, device=src.device)
     if workspace is None:
         workspace = torch.empty(fbsr_stats_workspace_bytes(), dtype=torch.uint8, device=src.device)
     with torch.cuda.device(src.device):
         _check(_L.fbsr_round_stats(_dev(src, torch.float32, "src"), po, n, _fmt(fmt), _var(variant), k_bits, seed,
-                                   offset, scale, group_size, ctypes.c_void_p(ge.data_ptr()),
-                                   ctypes.c_void_p(ge2.data_ptr()), ctypes.c_void_p(total.data_ptr()),
+                                   offset, scale, group_size, ctypes.c_void_p(ge.data_ptr()) if ge is not None else None,
+                                   ctypes.c_void_p(ge2.data_ptr()) if ge2 is not None else None,
+                                   ctypes.c_void_p(total.data_ptr()),
                                    ctypes.c_void_p(workspace.data_ptr()), workspace.numel(), _stream(src)),
                "fbsr_round_stats")
+    if not read_back:
+        return out, total, (ge[:groups] if ge is not None else None), (ge2[:groups] if ge2 is not None else None)
     st = FbsrStats.from_buffer_copy(total.cpu().numpy().tobytes())
     return out, {name: getattr(st, name) for name, _ in FbsrStats._fields_}, ge[:groups], ge2[:groups]
 

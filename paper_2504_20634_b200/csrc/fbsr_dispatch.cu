@@ -67,23 +67,37 @@ template <int SRC> inline LpSrcOp<SRC> op_advance(LpSrcOp<SRC> o, size_t h)
     o.src = static_cast<const uint16_t*>(o.src) + h; return o;
 }
 
-struct Plan { size_t head, n_tiles, tail_begin; };
+struct Plan { size_t head, n_tiles, tail_begin; bool aligned; };
+
+// Ops that also have the staged kernel, which takes pointers of any alignment (generated draws only).
+template <class Op, bool BITS> struct HasStaged { static constexpr bool value = false; };
+template <> struct HasStaged<RoundOp, false> { static constexpr bool value = true; };
 
 template <class Op, int VAR, int K, bool BITS>
 int launch_tiles(const Op& op, const CallArgs& a, const Plan& p)
 {
     using T = Tile<K, Op::OCTETS>;
-    auto kern = tile_kernel<Op, FMT, VAR, K, BITS>;
-    // One tile per warp, CTAs handed out by the hardware scheduler.  A persistent grid with a static
-    // tile stride measured 5-10 % slower here: multiprocessors do not all see the same memory
-    // bandwidth, and a static split makes the whole launch wait for the slowest of them.
     const uint32_t tail_count = (uint32_t)(a.n - p.tail_begin);          // < one tile; served by an extra CTA
-    const uint64_t want = (p.n_tiles + WARPS_PER_CTA - 1) / WARPS_PER_CTA;
-    const unsigned grid = (unsigned)(want < 0x7FFFFFF0ull ? want : 0x7FFFFFF0ull) + (tail_count ? 1u : 0u);
     const Op adv = op_advance(op, p.head);
     void* dst = static_cast<char*>(a.dst) + p.head * CODE_BYTES;
     const uint64_t call0 = BITS ? 0 : (a.offset + p.head) / T::E;
     const uint32_t* words = BITS ? a.words + p.head / T::DPW : nullptr;
+    if constexpr (HasStaged<Op, BITS>::value) {
+        if (!p.aligned) {
+            const uint64_t want = (p.n_tiles + STAGED_WARPS - 1) / STAGED_WARPS;
+            const unsigned grid = (unsigned)(want < 0x7FFFFFF0ull ? want : 0x7FFFFFF0ull) + (tail_count ? 1u : 0u);
+            staged_tile_kernel<FMT, VAR, K, BITS><<<grid, STAGED_THREADS, 0, a.stream>>>(
+                adv, dst, p.n_tiles, call0, (uint32_t)a.seed, (uint32_t)(a.seed >> 32), words, tail_count);
+            count_launch();
+            return 0;
+        }
+    }
+    auto kern = tile_kernel<Op, FMT, VAR, K, BITS>;
+    // One tile per warp, CTAs handed out by the hardware scheduler.  A persistent grid with a static
+    // tile stride measured 5-10 % slower here: multiprocessors do not all see the same memory
+    // bandwidth, and a static split makes the whole launch wait for the slowest of them.
+    const uint64_t want = (p.n_tiles + WARPS_PER_CTA - 1) / WARPS_PER_CTA;
+    const unsigned grid = (unsigned)(want < 0x7FFFFFF0ull ? want : 0x7FFFFFF0ull) + (tail_count ? 1u : 0u);
     kern<<<grid, CTA_THREADS, 0, a.stream>>>(adv, dst, p.n_tiles, call0, (uint32_t)a.seed,
                                              (uint32_t)(a.seed >> 32), words, tail_count);
     count_launch();
@@ -115,12 +129,12 @@ template <class Op, int K, bool BITS>
 Plan make_plan(const Op& op, const CallArgs& a)
 {
     using T = Tile<K, Op::OCTETS>;
-    Plan p{0, 0, 0};
+    Plan p{0, 0, 0, false};
     const uint64_t off = BITS ? 0 : a.offset;
     const size_t head = (size_t)((T::ELEMS - off % T::ELEMS) % T::ELEMS);
     const size_t dst_align = (CODE_BYTES == 2 ? 16 : 8) * Op::OCTETS;      // one vector store per lane-row
-    if (head < a.n && op_aligned(op, head) &&
-        aligned(static_cast<char*>(a.dst) + head * CODE_BYTES, dst_align)) {
+    p.aligned = op_aligned(op, head) && aligned(static_cast<char*>(a.dst) + head * CODE_BYTES, dst_align);
+    if (head < a.n && (p.aligned || HasStaged<Op, BITS>::value)) {
         p.head = head;
         p.n_tiles = (a.n - head) / T::ELEMS;
     }
@@ -221,12 +235,13 @@ int run_stats(const CallArgs& a)
     const RoundOp op{a.src, a.scale};
     StatsAcc* slots = static_cast<StatsAcc*>(a.partials);
     int n_slots = 0;
-    const Plan p = a.ovf_ieee ? Plan{0, 0, 0} : make_plan<RoundOp, K, false>(op, a);
-    if (p.n_tiles > 0) {
+    const Plan p = a.ovf_ieee ? Plan{0, 0, 0, false} : make_plan<RoundOp, K, false>(op, a);
+    if (p.n_tiles > 0 && p.aligned) {
         using T = Tile<K, 1>;
         const uint64_t want = (p.n_tiles + WARPS_PER_CTA - 1) / WARPS_PER_CTA;
         const unsigned grid = (unsigned)(want < (uint64_t)STATS_TILE_GRID ? want : (uint64_t)STATS_TILE_GRID);
-        stats_tile_kernel<FMT, VAR, K><<<grid, CTA_THREADS, 0, a.stream>>>(
+        auto kern = a.group_size ? stats_tile_kernel<FMT, VAR, K, true> : stats_tile_kernel<FMT, VAR, K, false>;
+        kern<<<grid, CTA_THREADS, 0, a.stream>>>(
             a.src + p.head, a.scale, static_cast<char*>(a.dst) + p.head * CODE_BYTES, p.n_tiles, p.head,
             (a.offset + p.head) / T::E, (uint32_t)a.seed, (uint32_t)(a.seed >> 32), a.group_size, a.gsum_e, a.gsum_e2,
             slots);

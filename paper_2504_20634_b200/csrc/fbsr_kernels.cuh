@@ -741,6 +741,155 @@ tile_kernel(const Op op, void* __restrict__ dst, const uint64_t n_tiles, const u
     }
 }
 
+// ---------------------------------------------------------------------------- the bandwidth kernel, any alignment
+// fbsr_round for pointers that are only element-aligned (a slice of a tensor, a packed parameter buffer).  The
+// tile grid is fixed by `offset` (a tile is a whole number of generator calls), so no peeling can also align the
+// two pointers; instead a warp stages its tile through shared memory:
+//   in   element j of the tile is copied to shared word j by 4-byte asynchronous copies, lane-consecutive, so a
+//        warp instruction still reads 128 contiguous bytes of global memory whatever the pointer's alignment, and
+//        the whole tile is in flight at once; a lane then takes its 8 consecutive values with two 128-bit reads;
+//   out  the packed codes go to shared memory (over values already consumed), and are written out as
+//        4-byte words aligned in GLOBAL memory: word m is funnelled out of two neighbouring shared words by a
+//        byte permute whose selector is the pointer's misalignment; the few bytes before the first and after the
+//        last aligned word of the tile are stored one code at a time (the neighbouring tile writes the rest of
+//        that word).
+// Rounding, draws and the treatment of special values are those of tile_kernel.
+constexpr int STAGED_WARPS = 4;                          // keeps the static shared memory of every k under 48 KB
+constexpr int STAGED_THREADS = STAGED_WARPS * 32;
+
+__device__ __forceinline__ void copy_async_4(void* smem_dst, const void* gmem_src)
+{
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gmem_src) : "memory");
+}
+
+template <int FMT, int VAR, int K, bool BITS>
+__global__ void __launch_bounds__(STAGED_THREADS, 4)
+staged_tile_kernel(const RoundOp op, void* __restrict__ dst, const uint64_t n_tiles, const uint64_t call0,
+                   const uint32_t k0, const uint32_t k1, const uint32_t* __restrict__ words, const uint32_t tail_count)
+{
+    using T = Tile<K, 1>;
+    constexpr bool DRAWS = VAR < RTNE;
+    constexpr int CB = Format<FMT>::K / 8;
+    const uint32_t first_tile_cta = tail_count ? 1u : 0u;
+    if (tail_count && blockIdx.x == 0) {
+        // the elements after the last whole tile, one per thread and step, as in tile_kernel
+        const size_t tail_begin = (size_t)n_tiles * T::ELEMS;
+        for (uint32_t i = threadIdx.x; i < tail_count; i += STAGED_THREADS) {
+            const size_t p = tail_begin + i;
+            const uint32_t j = (uint32_t)(p % T::E);
+            uint32_t word = 0u;
+            if constexpr (!DRAWS) {
+            } else if constexpr (BITS) {
+                word = words[p / T::DPW];
+            } else {
+                const uint4 o = philox_block(call0 + p / T::E, k0, k1);
+                const uint32_t ws = j / T::DPW;
+                word = ws == 0 ? o.x : ws == 1 ? o.y : ws == 2 ? o.z : o.w;
+            }
+            const uint32_t n = (word >> ((j % T::DPW) * K)) & T::MASK;
+            store_code1<FMT>(dst, p, round_core<FMT, false>(op.scalar(p), n, VAR, K, nullptr));
+        }
+        return;
+    }
+    constexpr bool OWN_CALL = (T::DPW == 2) && !BITS;
+    constexpr int OUT_WORDS = T::ELEMS * CB / 4;
+    // the packed codes of row j (at most half as many bytes as its values) overwrite the front of the same buffer:
+    // bytes [0, 256 (j + 1) CB) only ever held rows 0..j, which the warp has already taken into registers
+    static_assert(OUT_WORDS + 1 <= T::ELEMS, "the codes and the funnel's look-ahead word fit in the input buffer");
+    __shared__ __align__(16) float in_buf[STAGED_WARPS][T::ELEMS];
+    __shared__ __align__(16) uint32_t wordbuf[STAGED_WARPS][OWN_CALL ? 4 : (BITS ? T::WORDS + 4 : T::BUFFER_WORDS)];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    float* in = in_buf[warp];
+    uint32_t* ob = reinterpret_cast<uint32_t*>(in);
+    uint32_t* wb = wordbuf[warp];
+    constexpr int ROWS = T::ELEMS / ROW_ELEMS;
+    constexpr int WPO = WordsPerOctet<FMT>::value;
+
+    for (uint64_t tile = (uint64_t)(blockIdx.x - first_tile_cta) * STAGED_WARPS + warp; tile < n_tiles;
+         tile += (uint64_t)(gridDim.x - first_tile_cta) * STAGED_WARPS) {
+        const size_t e0 = (size_t)tile * T::ELEMS;
+        const uint64_t tile_call0 = call0 + tile * T::CALLS;
+        const float* src = op.src + e0;
+#pragma unroll
+        for (int j = 0; j < T::ELEMS / 32; ++j) copy_async_4(in + j * 32 + lane, src + j * 32 + lane);
+        asm volatile("cp.async.commit_group;" ::: "memory");
+
+        // the generator calls run while the copies are in flight
+        if constexpr (!DRAWS) {
+        } else if constexpr (BITS) {
+            const uint32_t* src_words = words + tile * T::WORDS;
+#pragma unroll
+            for (int j = 0; j < T::WORDS / 32; ++j) wb[j * 32 + lane] = __ldg(src_words + j * 32 + lane);
+        } else if constexpr (!OWN_CALL) {
+#pragma unroll
+            for (int j = 0; j < (T::CALLS + 31) / 32; ++j) {
+                const int c = j * 32 + lane;
+                if (T::CALLS % 32 == 0 || c < T::CALLS)
+                    Draws8<K>::store_call(wb + Draws8<K>::WORDS_PER_CALL * c, philox_block(tile_call0 + c, k0, k1));
+            }
+        }
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
+        __syncwarp();
+
+#pragma unroll
+        for (int j = 0; j < ROWS; ++j) {
+            const int p0 = j * ROW_ELEMS + lane * 8;
+            RoundOp::Regs regs;
+            regs.x.a = *reinterpret_cast<const float4*>(in + p0);
+            regs.x.b = *reinterpret_cast<const float4*>(in + p0 + 4);
+            __syncwarp();                                    // every lane holds its values before codes are written over them
+            float y[8];
+            op.finish(e0 + p0, regs, y);
+            Draws8<K> d;
+            if constexpr (!DRAWS) {
+            } else if constexpr (OWN_CALL) {
+                d.from_call(philox_block(tile_call0 + p0 / 8, k0, k1));
+            } else if constexpr (BITS) {
+                d.from_stream(wb, p0);
+            } else {
+                d.from_normalised(wb, p0);
+            }
+            uint32_t t[8], packed[WPO];
+            const bool redo = round_row_fast<FMT, VAR, K>(y, d, t);
+            if (!redo) {
+                pack_row_fast<FMT>(t, y, packed);
+            } else {
+                uint32_t c[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i)
+                    c[i] = round_core<FMT, false>(op.exact_bits(regs, i, y[i]), d.template at<0>(i), VAR, K, nullptr);
+                pack_codes8<FMT>(c, packed);
+            }
+            if constexpr (WPO == 4) *reinterpret_cast<uint4*>(ob + p0 / 2) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+            else *reinterpret_cast<uint2*>(ob + p0 / 4) = make_uint2(packed[0], packed[1]);
+        }
+        __syncwarp();
+
+        // write-out: 4-byte words aligned in global memory
+        char* g = static_cast<char*>(dst) + e0 * CB;
+        const uint32_t head_b = (4u - (uint32_t)(reinterpret_cast<uintptr_t>(g) & 3u)) & 3u;      // bytes before the first aligned word
+        const uint32_t n_words = head_b ? OUT_WORDS - 1 : OUT_WORDS;
+        const uint32_t selector = 0x3210u + 0x1111u * head_b;
+        uint32_t* gw = reinterpret_cast<uint32_t*>(g + head_b);
+#pragma unroll 4
+        for (uint32_t m = lane; m < n_words; m += 32) FBSR_STORE(gw + m, __byte_perm(ob[m], ob[m + 1], selector));
+        if (head_b) {
+            // the codes before the first aligned word and after the last one
+            const uint32_t head_codes = head_b / CB, tail_codes = (4u - head_b) / CB;
+            const unsigned char* bytes = reinterpret_cast<const unsigned char*>(ob);
+            if ((uint32_t)lane < head_codes) {
+                if constexpr (CB == 2) reinterpret_cast<uint16_t*>(g)[lane] = reinterpret_cast<const uint16_t*>(bytes)[lane];
+                else reinterpret_cast<uint8_t*>(g)[lane] = bytes[lane];
+            } else if ((uint32_t)lane < head_codes + tail_codes) {
+                const uint32_t i = T::ELEMS - tail_codes + ((uint32_t)lane - head_codes);
+                if constexpr (CB == 2) reinterpret_cast<uint16_t*>(g)[i] = reinterpret_cast<const uint16_t*>(bytes)[i];
+                else reinterpret_cast<uint8_t*>(g)[i] = bytes[i];
+            }
+        }
+        __syncwarp();                                        // the buffers are rewritten by the next tile
+    }
+}
+
 // ---------------------------------------------------------------------------- statistics
 struct StatsAcc {
     unsigned long long n_finite, n_up, n_nan, n_inf, n_sat;
@@ -897,13 +1046,150 @@ __device__ __forceinline__ bool stats_element(const uint32_t ybits, const uint32
     return true;
 }
 
+// ---------------------------------------------------------------------------- statistics on whole tiles
+// Integer form of the error sums.  With delta~ = d / 2^U (d an integer) and up in {0, 1}, e = up - delta~ gives
+//   sum e    = (n_up 2^U - sum d) / 2^U
+//   sum |e|  = (sum d - 2 sum_{up} d + n_up 2^U) / 2^U
+//   sum e^2  = (sum d^2 + n_up 2^(2U) - 2^(U+1) sum_{up} d) / 2^(2U)
+//   sum s e  = sum e - 2 (n_{up, y<0} 2^U - sum_{y<0} d) / 2^U          (s = sign of y)
+// so a thread only adds d, d^2 and a few masked copies of d per element, all exact in 64-bit integers, and turns
+// them into binary64 once.  U = 16 for bfloat16 (the excess bits are always the low half of the pattern) and 23
+// for the other formats, which covers every element with at most 23 excess bits: the target's normal range,
+// its subnormal range and the binade below.  An element with more excess bits ("deep": a magnitude below a
+// quarter of the smallest subnormal, so floor(sigma~) = 0 and delta~ = sigma~ < 1, an exact binary32 product)
+// enters the integer sums with d = 0 and adds its delta~ to the same four sums kept in binary64 beside them.
+// NaN and Inf send the lane's octet through stats_element() instead.
+template <int FMT> struct StatsFixed {
+    using F = Format<FMT>;
+    static constexpr int U = FMT == BF16 ? 16 : 23;
+    static constexpr int SH0 = 24 - F::P;
+    // smallest pattern with at most 23 excess bits: biased exponent EMINB - P + 1
+    static constexpr uint32_t DEEP_BITS = FMT == BF16 ? 0u : (uint32_t)(F::EMINB - F::P + 1) << 23;
+};
+
+struct StatsInt {                        // one lane's integer sums, units of 2^-U
+    unsigned long long d, up_d, neg_d, d2;          // sum d, over rounded-up elements, over negative elements, sum d^2
+    uint32_t d_tile, up_d_tile, neg_d_tile;         // the first three over the current tile (at most 48 elements: no overflow)
+    uint32_t counts;                    // rounded up: low half; rounded up and negative: high half (unpacked every tile)
+    uint32_t n_sat;
+};
+
+struct StatsDeep { double d, up_d, neg_d, d2; };      // the same sums of delta~ over the deep elements
+
+__device__ __forceinline__ uint32_t shl_clamped(uint32_t x, int s)
+{
+    uint32_t r;
+    asm("shl.b32 %0, %1, %2;" : "=r"(r) : "r"(x), "r"((uint32_t)s));   // amounts above 31 give 0
+    return r;
+}
+
+// One SR-rounded (or saturated) finite element: y the value, t the word left by round_row_fast.  The masked
+// sums are written as 32-bit multiply-adds (`one` is 1, unknown to the compiler) so that they run on the
+// multiplier pipe: the integer pipe is what bounds this kernel.  (64-bit widening multiply-adds measured slower.)
+template <int FMT>
+__device__ __forceinline__ void stats_fixed_element(const float y, const uint32_t t, const uint32_t one, StatsInt& s,
+                                                    StatsDeep& deep)
+{
+    using F = Format<FMT>;
+    using X = StatsFixed<FMT>;
+    const uint32_t yb = __float_as_uint(y);
+    const uint32_t neg = yb >> 31;
+    uint32_t d, up;
+    if constexpr (FMT == BF16) {
+        d = yb & 0xFFFFu;
+        up = ((t ^ yb) >> 16) & 1u;                                      // the code's lowest bit flips iff a carry came in
+    } else {
+        const uint32_t ab = yb & 0x7FFFFFFFu;
+        const bool sat = ab > F::MAXBITS;                               // counted, and never rounded up: d = 0
+        s.n_sat += sat ? 1u : 0u;
+        // left-align the excess bits: 32 - sh = min(32 - SH0, eb + 32 - SH0 - EMINB); a shift below 9 (more than
+        // 23 excess bits) leaves exponent bits in the way, so those elements take d = 0 here
+        const int s8 = min(32 - X::SH0, (int)(ab >> 23) + (32 - X::SH0 - F::EMINB));
+        const bool is_deep = (ab - 1u) < (X::DEEP_BITS - 1u);           // zero is not deep: all its terms are 0
+        d = (is_deep || sat) ? 0u : shl_clamped(ab, s8) >> 9;
+        // floor code from the rescaled pattern, as in the row rounder
+        const float rescale = __uint_as_float((uint32_t)(128 - F::EMINB) << 23);
+        const uint32_t u = min(__float_as_uint(__fmul_rz(fabsf(y), rescale)), F::MAXCODE << X::SH0);
+        up = ((t ^ (u << (32 - F::K - X::SH0))) >> (32 - F::K)) & 1u;    // lowest bit of the code against the floor's
+        if (is_deep) {
+            // sigma~ = |y| 2^(P - 1 - emin), exact
+            const double dl = (double)__fmul_rn(fabsf(y), __uint_as_float((uint32_t)(F::P - 1 + 254 - F::EMINB) << 23));
+            deep.d += dl;
+            deep.d2 = fma(dl, dl, deep.d2);
+            if (up) deep.up_d += dl;
+            if (neg) deep.neg_d += dl;
+        }
+    }
+    s.d_tile += d;
+    s.d2 += (unsigned long long)d * d;
+    s.up_d_tile += up * d;
+    s.neg_d_tile += neg * d;
+    if constexpr (F::K == 16) s.counts += up + ((up & neg) << 16);
+    else s.counts += up * (neg * 65536u + one);
+}
+
+// One lane-octet element by element in binary64 (the octets that hold NaN or Inf or, with group sums, a group
+// boundary): rounds and stores its 8 codes and adds their statistics to
+// *sums.  Kept out of line, with the binary64 sums in local memory, so that neither takes registers from the tile
+// loop; it reads its inputs again.
+template <int FMT, bool GROUPS, int CALLER_VAR, int CALLER_K>         // one copy per calling kernel
+__device__ __noinline__ void stats_octet_general(StatsAcc* __restrict__ sums, const float* __restrict__ src8, const float scale,
+                                                 const uint4 n_lo, const uint4 n_hi, const int variant, const int k,
+                                                 void* __restrict__ dst8, const uint64_t i0, const uint64_t group_size,
+                                                 double* __restrict__ gsum_e, double* __restrict__ gsum_e2)
+{
+    const uint32_t n[8] = {n_lo.x, n_lo.y, n_lo.z, n_lo.w, n_hi.x, n_hi.y, n_hi.z, n_hi.w};
+    using F = Format<FMT>;
+    constexpr uint32_t MAG = (1u << (F::K - 1)) - 1u;
+    StatsAcc acc = *sums;
+    float x[8], y[8];
+    unpack(load_f8(src8), x);
+#pragma unroll
+    for (int c = 0; c < 8; ++c) y[c] = __fmul_rn(x[c], scale);
+    uint32_t codes[8], packed[WordsPerOctet<FMT>::value];
+#pragma unroll
+    for (int c = 0; c < 8; ++c) {
+        const uint32_t bits = y[c] != y[c] ? __float_as_uint(x[c]) : __float_as_uint(y[c]);   // a NaN keeps the input's sign
+        codes[c] = round_core<FMT, false>(bits, n[c], variant, k, nullptr);
+    }
+    pack_codes8<FMT>(codes, packed);
+    store_words<WordsPerOctet<FMT>::value>(dst8, packed);
+    // group sums are flushed where the run of 8 crosses a group boundary
+    uint64_t grp = 0, grp_end = ~0ull;
+    double ge = 0.0, ge2 = 0.0;
+    if (GROUPS) { grp = i0 / group_size; grp_end = (grp + 1) * group_size; }
+#pragma unroll
+    for (int c = 0; c < 8; ++c) {
+        uint32_t up = 0;
+        double e = 0.0;
+        if (stats_element<FMT>(__float_as_uint(y[c]), codes[c] & MAG, acc, e, up)) {
+            acc.n_finite += 1; acc.n_up += up;
+            acc.sum_e += e; acc.sum_e2 = fma(e, e, acc.sum_e2);
+            acc.sum_signed_e += (__float_as_uint(y[c]) >> 31) ? -e : e;
+            acc.sum_abs_e += fabs(e);
+            if (GROUPS) {
+                if (i0 + c >= grp_end) {
+                    if (ge != 0.0 || ge2 != 0.0) { atomicAdd(gsum_e + grp, ge); atomicAdd(gsum_e2 + grp, ge2); }
+                    ge = 0.0; ge2 = 0.0;
+                    grp = (i0 + c) / group_size; grp_end = (grp + 1) * group_size;
+                }
+                ge += e; ge2 = fma(e, e, ge2);
+            }
+        }
+    }
+    if (GROUPS && (ge != 0.0 || ge2 != 0.0)) { atomicAdd(gsum_e + grp, ge); atomicAdd(gsum_e2 + grp, ge2); }
+    *sums = acc;
+}
+
 // Statistics on whole tiles: the rounding of the bandwidth kernel (generator calls shared through the warp's
-// buffer, row rounder, packed stores) followed, per element, by stats_element() on the value and its code.
-// A capped grid walks the tiles with a fixed stride, so each thread adds its elements in a fixed order and
-// leaves one partial per CTA: the totals are reproducible bit for bit.
+// buffer, row rounder, packed stores) followed by the integer sums above; octets holding NaN or Inf (and, with
+// group sums, octets that straddle a group boundary) go through stats_element() in binary64.  A capped grid walks the tiles with a fixed stride, so each thread adds its
+// elements in a fixed order and leaves one partial per CTA: the totals are reproducible bit for bit.
 // first_index: index within the call of element 0 (for the group sums).
-template <int FMT, int VAR, int K>
-__global__ void __launch_bounds__(CTA_THREADS, 3)
+constexpr int STATS_MIN_CTAS = 3;                        // resident CTAs the compiler must allow (caps the registers at 80)
+constexpr int STATS_ROWS_IN_FLIGHT = 2;                  // rows whose loads are outstanding per warp
+template <int FMT, int VAR, int K, bool GROUPS>
+__global__ void __launch_bounds__(CTA_THREADS, STATS_MIN_CTAS)
 stats_tile_kernel(const float* __restrict__ src, const float scale, void* __restrict__ dst, const uint64_t n_tiles,
                   const uint64_t first_index, const uint64_t call0, const uint32_t k0, const uint32_t k1,
                   const uint64_t group_size, double* __restrict__ gsum_e, double* __restrict__ gsum_e2,
@@ -911,23 +1197,27 @@ stats_tile_kernel(const float* __restrict__ src, const float scale, void* __rest
 {
     using T = Tile<K, 1>;
     using F = Format<FMT>;
+    using X = StatsFixed<FMT>;
     constexpr bool DRAWS = VAR < RTNE;
     constexpr bool OWN_CALL = T::DPW == 2;
     constexpr int ROWS = T::ELEMS / ROW_ELEMS;
     constexpr int WPO = WordsPerOctet<FMT>::value;
-    constexpr uint32_t MAG = (1u << (F::K - 1)) - 1u;
+    constexpr int U = X::U;
     __shared__ __align__(16) uint32_t wordbuf[WARPS_PER_CTA][OWN_CALL ? 4 : T::BUFFER_WORDS];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     uint32_t* wb = wordbuf[warp];
-    StatsAcc acc;
+    StatsAcc acc;                                            // binary64 side: the octets done element by element
     stats_zero(acc);
+    StatsInt tot = {0ull, 0ull, 0ull, 0ull, 0u, 0u, 0u, 0u, 0u};
+    uint32_t n_up = 0, n_up_neg = 0, fast_octets = 0;       // a thread sees far fewer than 2^32 elements
+    StatsDeep deep = {0.0, 0.0, 0.0, 0.0};
+    const uint32_t one = min(blockDim.x, 1u);
 
     for (uint64_t tile = (uint64_t)blockIdx.x * WARPS_PER_CTA + warp; tile < n_tiles;
          tile += (uint64_t)gridDim.x * WARPS_PER_CTA) {
         const size_t e0 = (size_t)tile * T::ELEMS;
         const uint64_t tile_call0 = call0 + tile * T::CALLS;
-        // rows are loaded two at a time: the statistics need the registers that deeper prefetching would take
-        constexpr int BATCH = 2;
+        constexpr int BATCH = STATS_ROWS_IN_FLIGHT < ROWS ? STATS_ROWS_IN_FLIGHT : ROWS;
         F8 regs[BATCH];
 #pragma unroll
         for (int j = 0; j < BATCH; ++j) regs[j] = load_f8_stream(src + e0 + j * ROW_ELEMS + lane * 8);
@@ -955,61 +1245,68 @@ stats_tile_kernel(const float* __restrict__ src, const float scale, void* __rest
             } else {
                 d.from_normalised(wb, p0);
             }
-            uint32_t t[8], codes[8], packed[WPO];
+            uint32_t t[8], packed[WPO];
             const bool redo = round_row_fast<FMT, VAR, K>(y, d, t);
-            if (!redo) {
-                pack_row_fast<FMT>(t, y, packed);
-#pragma unroll
-                for (int c = 0; c < 8; ++c) codes[c] = (t[c] >> (32 - F::K)) & MAG;
-            } else {
-#pragma unroll
-                for (int c = 0; c < 8; ++c) {
-                    const uint32_t bits = y[c] != y[c] ? __float_as_uint(x[c]) : __float_as_uint(y[c]);   // a NaN keeps the input's sign
-                    codes[c] = round_core<FMT, false>(bits, d.template at<0>(c), VAR, K, nullptr);
-                }
-                pack_codes8<FMT>(codes, packed);
-#pragma unroll
-                for (int c = 0; c < 8; ++c) codes[c] &= MAG;
-            }
-            store_words<WPO>(static_cast<char*>(dst) + (e0 + p0) * (F::K / 8), packed);
-
-            // statistics of the row's 8 elements; group sums are flushed where a lane's run crosses a group
             const uint64_t i0 = first_index + e0 + p0;
-            uint64_t grp = 0, grp_end = ~0ull;
-            double ge = 0.0, ge2 = 0.0;
-            if (group_size) { grp = i0 / group_size; grp_end = (grp + 1) * group_size; }
-            // the row's eight errors first, then their sums as short trees in a fixed order (no long dependent chain)
-            double e[8];
-            uint32_t n_fin = 0, n_up = 0;
+            bool fast = !redo;
+            if constexpr (GROUPS) fast &= i0 / group_size == (i0 + 7) / group_size;
+            if (fast) {
+                pack_row_fast<FMT>(t, y, packed);
+                StatsInt os = {0ull, 0ull, 0ull, 0ull, 0u, 0u, 0u, 0u, 0u};
+                StatsInt& s = GROUPS ? os : tot;
+                StatsDeep od = {0.0, 0.0, 0.0, 0.0};
+                StatsDeep& dp = GROUPS ? od : deep;
 #pragma unroll
-            for (int c = 0; c < 8; ++c) {
-                uint32_t up = 0;
-                e[c] = 0.0;
-                if (stats_element<FMT>(__float_as_uint(y[c]), codes[c], acc, e[c], up)) {
-                    n_fin += 1; n_up += up;
-                    if (group_size) {
-                        while (i0 + c >= grp_end) {
-                            if (ge != 0.0 || ge2 != 0.0) { atomicAdd(gsum_e + grp, ge); atomicAdd(gsum_e2 + grp, ge2); }
-                            ge = 0.0; ge2 = 0.0;
-                            grp = (i0 + c) / group_size; grp_end = (grp + 1) * group_size;
-                        }
-                        ge += e[c]; ge2 = fma(e[c], e[c], ge2);
+                for (int c = 0; c < 8; ++c) stats_fixed_element<FMT>(y[c], t[c], one, s, dp);
+                fast_octets += 1;
+                if constexpr (GROUPS) {
+                    // the octet lies in one group: e and e^2 summed exactly, then one pair of atomics
+                    const long long oct_up = os.counts & 0xFFFFu;
+                    const long long ge = (oct_up << U) - (long long)os.d_tile;
+                    const long long ge2 = (long long)os.d2 + (oct_up << (2 * U)) - ((long long)os.up_d_tile << (U + 1));
+                    if (ge != 0 || ge2 != 0 || od.d != 0.0) {
+                        const uint64_t grp = i0 / group_size;
+                        atomicAdd(gsum_e + grp, (double)ge * __hiloint2double((1023 - U) << 20, 0) - od.d);
+                        atomicAdd(gsum_e2 + grp, (double)ge2 * __hiloint2double((1023 - 2 * U) << 20, 0) + (od.d2 - 2.0 * od.up_d));
                     }
+                    deep.d += od.d; deep.up_d += od.up_d; deep.neg_d += od.neg_d; deep.d2 += od.d2;
+                    tot.d_tile += os.d_tile; tot.up_d_tile += os.up_d_tile; tot.neg_d_tile += os.neg_d_tile; tot.d2 += os.d2;
+                    tot.counts += os.counts; tot.n_sat += os.n_sat;
                 }
-            }
-            if (group_size && (ge != 0.0 || ge2 != 0.0)) { atomicAdd(gsum_e + grp, ge); atomicAdd(gsum_e2 + grp, ge2); }
-            acc.n_finite += n_fin; acc.n_up += n_up;
-            double s[8];
+                store_words<WPO>(static_cast<char*>(dst) + (e0 + p0) * (F::K / 8), packed);
+            } else {
+                uint32_t n[8];
 #pragma unroll
-            for (int c = 0; c < 8; ++c) s[c] = (__float_as_uint(y[c]) >> 31) ? -e[c] : e[c];
-            acc.sum_e += ((e[0] + e[1]) + (e[2] + e[3])) + ((e[4] + e[5]) + (e[6] + e[7]));
-            acc.sum_signed_e += ((s[0] + s[1]) + (s[2] + s[3])) + ((s[4] + s[5]) + (s[6] + s[7]));
-            acc.sum_abs_e += ((fabs(e[0]) + fabs(e[1])) + (fabs(e[2]) + fabs(e[3]))) +
-                             ((fabs(e[4]) + fabs(e[5])) + (fabs(e[6]) + fabs(e[7])));
-            acc.sum_e2 += (fma(e[0], e[0], e[1] * e[1]) + fma(e[2], e[2], e[3] * e[3])) +
-                          (fma(e[4], e[4], e[5] * e[5]) + fma(e[6], e[6], e[7] * e[7]));
+                for (int c = 0; c < 8; ++c) n[c] = DRAWS ? d.template at<0>(c) : 0u;
+                stats_octet_general<FMT, GROUPS, VAR, K>(&acc, src + e0 + p0, scale, make_uint4(n[0], n[1], n[2], n[3]),
+                                                 make_uint4(n[4], n[5], n[6], n[7]), VAR, K,
+                                                 static_cast<char*>(dst) + (e0 + p0) * (F::K / 8), i0, group_size, gsum_e, gsum_e2);
+            }
         }
+        // at most 48 elements a tile: the 32-bit sums and the packed counts are folded in before they can overflow
+        tot.d += tot.d_tile; tot.up_d += tot.up_d_tile; tot.neg_d += tot.neg_d_tile;
+        tot.d_tile = tot.up_d_tile = tot.neg_d_tile = 0u;
+        n_up += tot.counts & 0xFFFFu; n_up_neg += tot.counts >> 16; tot.counts = 0u;
         if constexpr (DRAWS && !OWN_CALL) __syncwarp();      // the buffer is rewritten by the next tile
+    }
+    // the thread's integer sums, exact, turned into binary64 once
+    {
+        const double unit = __hiloint2double((1023 - U) << 20, 0), unit2 = __hiloint2double((1023 - 2 * U) << 20, 0);
+        const unsigned long long ups = n_up, ups_neg = n_up_neg;
+        const long long se = (long long)(ups << U) - (long long)tot.d;
+        const long long sneg = (long long)(ups_neg << U) - (long long)tot.neg_d;
+        const unsigned long long sabs = tot.d - 2ull * tot.up_d + (ups << U);
+        const unsigned __int128 s2 = (unsigned __int128)tot.d2 + ((unsigned __int128)ups << (2 * U)) -
+                                     ((unsigned __int128)tot.up_d << (U + 1));
+        acc.n_finite += 8ull * fast_octets - tot.n_sat;
+        acc.n_up += ups;
+        acc.n_sat += tot.n_sat;
+        // deep elements: e = up - delta~ with the integer sums holding up alone
+        acc.sum_e += (double)se * unit - deep.d;
+        acc.sum_signed_e += (double)(se - 2 * sneg) * unit - (deep.d - 2.0 * deep.neg_d);
+        acc.sum_abs_e += (double)sabs * unit + (deep.d - 2.0 * deep.up_d);
+        acc.sum_e2 += ((double)(unsigned long long)(s2 >> 64) * 18446744073709551616.0 + (double)(unsigned long long)s2) * unit2 +
+                      (deep.d2 - 2.0 * deep.up_d);
     }
     stats_cta_reduce(acc);
     if (threadIdx.x == 0) partials[blockIdx.x] = acc;

@@ -25,16 +25,26 @@ def main():
     ap.add_argument("--log2n", type=int, default=26)
     ap.add_argument("--iters", type=int, default=5)
     ap.add_argument("--warmup", type=int, default=2)
+    ap.add_argument("--data", default="sweep", choices=["sweep", "fp8act"],
+                    help="sweep: N(0,1) x 2^U(-20,20); fp8act: Laplace activations with amax scaling and injected outliers (8-bit formats)")
+    ap.add_argument("--scale", type=float, default=1.0, help="per-tensor scale for --op round / stats on the sweep data")
+    ap.add_argument("--misalign", type=int, default=0, help="start the source this many elements off its allocation (--op round)")
     args = ap.parse_args()
 
     n = 1 << args.log2n
     dev = torch.device("cuda", 0)
-    x = workloads.bandwidth_sweep(n, seed=1234, device=dev)
+    scale = args.scale
+    if args.data == "fp8act":
+        x, scale = workloads.fp8_activations(args.fmt, rows=n // 32768, cols=32768, device=dev)
+    elif args.misalign:
+        x = workloads.bandwidth_sweep(n + args.misalign, seed=1234, device=dev)[args.misalign:]
+    else:
+        x = workloads.bandwidth_sweep(n, seed=1234, device=dev)
     code_bytes = 2 if args.fmt in ("bf16", "fp16") else 1
     out = torch.empty(n, dtype=fbsr.CODE_DTYPE[args.fmt], device=dev)
     if args.op == "round":
         bytes_per_elem = 4 + code_bytes
-        run = lambda s: fbsr.fbsr_round(x, args.fmt, args.variant, args.k, seed=1234, out=out)
+        run = lambda s: fbsr.fbsr_round(x, args.fmt, args.variant, args.k, seed=1234, scale=scale, out=out)
     elif args.op == "desc":
         # the same format, handed over as a run-time descriptor (general kernel)
         desc = fbsr.format_desc(*{"bf16": (16, 8, 127, 0x7F7F, 0x7F80, 0x7FC0, False),
@@ -67,7 +77,10 @@ def main():
         run = lambda s: fbsr.fbsr_round_bits(x, args.fmt, args.variant, args.k, words, out=out)
     elif args.op == "stats":
         bytes_per_elem = 4 + code_bytes
-        run = lambda s: fbsr.fbsr_round_stats(x, args.fmt, args.variant, args.k, seed=1234, out=out)
+        ws = torch.empty(fbsr.fbsr_stats_workspace_bytes(), dtype=torch.uint8, device=dev)
+        total = torch.empty(72, dtype=torch.uint8, device=dev)
+        run = lambda s: fbsr.fbsr_round_stats(x, args.fmt, args.variant, args.k, seed=1234, scale=scale, out=out,
+                                              workspace=ws, total=total, read_back=False)
     elif args.op == "accumulate":
         x.mul_(1e-3)
         out.copy_(workloads.accumulation_weights(n, device=dev) if args.fmt == "bf16" else torch.zeros_like(out))
@@ -93,7 +106,7 @@ def main():
     b.record()
     torch.cuda.synchronize()
     ms = a.elapsed_time(b) / args.iters
-    print(json.dumps({"op": args.op, "fmt": args.fmt, "variant": args.variant, "k": args.k, "n": n,
+    print(json.dumps({"op": args.op, "fmt": args.fmt, "variant": args.variant, "k": args.k, "n": n, "data": args.data, "scale": scale,
                       "ms_per_launch": ms, "GB/s": bytes_per_elem * n / (ms * 1e-3) / 1e9,
                       "Gelem/s": n / (ms * 1e-3) / 1e9}))
 

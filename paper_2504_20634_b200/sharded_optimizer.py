@@ -4,11 +4,12 @@ Every rank holds the whole low-precision copy of a flat parameter vector (what t
 passes read) but the binary32 master weights and Adam moments of its own shard only.  One step is
 
     1. (optional) reduce-scatter of the binary32 gradients, so that each rank gets the summed gradient
-       of its shard;
+       of its shard; the gradients live in a persistent padded buffer, so the step allocates nothing;
     2. the fused update of the shard: master weights and moments in place, and the stochastically rounded
        weights written straight into this rank's slice of the full low-precision buffer (the last line
        of Algorithm 1: the SR write lands in the buffer that the collective sends, no staging copy);
-    3. an in-place all-gather of that buffer over the process group (NCCL over NVLink on GPUs).
+    3. an in-place all-gather of that buffer over the process group (NCCL over NVLink on GPUs), issued
+       asynchronously so that it overlaps what the caller enqueues next.
 
 Draws are keyed by the global element index (``offset`` = start of the shard) and the seed of step t is
 ``seed + t``, so the gathered codes are bit-identical to one unsharded call on one GPU.  The only data
@@ -60,10 +61,15 @@ class ShardedLowPrecisionAdam:
         self.v = torch.zeros(self.n_own, **f32)
         self.lp_padded = torch.zeros(self.world * self.shard_len, dtype=code_dtype, device=self.device)
         self.step_count = 0
+        self._gather = None                # handle of the all-gather in flight
+        self._grad_padded = None           # made on first use by grad_buffer()
+        self._grad_shard = None
 
     @property
     def lp(self):
-        """The full low-precision parameter vector (n_total codes), valid on every rank after step()."""
+        """The full low-precision parameter vector (n_total codes), valid on every rank after step(); waits for
+        the all-gather in flight."""
+        self.wait_gather()
         return self.lp_padded[: self.n_total]
 
     def _own_slice(self):
@@ -79,22 +85,39 @@ class ShardedLowPrecisionAdam:
             raise ValueError("expected %d or %d elements" % (self.n_total, self.n_own))
         self.master.copy_(src)
 
-    def reduce_scatter_grad(self, full_grad):
-        """Sum the ranks' gradients of the full vector and return this rank's shard of the sum."""
-        if full_grad.numel() != self.n_total:
-            raise ValueError("full_grad must have n_total elements")
-        if self.world == 1:
-            return full_grad[self.start: self.end]
-        padded = torch.zeros(self.world * self.shard_len, dtype=torch.float32, device=self.device)
-        padded[: self.n_total].copy_(full_grad)
-        out = torch.empty(self.shard_len, dtype=torch.float32, device=self.device)
-        self.dist.reduce_scatter_tensor(out, padded, group=self.group)
-        return out[: self.n_own]
+    def grad_buffer(self):
+        """The persistent full-length gradient buffer (n_total binary32 values) that the backward pass may write
+        into directly; it is the front of a world x shard_len buffer whose tail stays zero, so that
+        reduce_scatter_grad() needs neither an allocation nor a padding copy."""
+        if self._grad_padded is None:
+            self._grad_padded = torch.zeros(self.world * self.shard_len, dtype=torch.float32, device=self.device)
+            self._grad_shard = torch.empty(self.shard_len, dtype=torch.float32, device=self.device)
+        return self._grad_padded[: self.n_total]
 
-    def step(self, grad_shard):
-        """One fused step on this rank's shard, then the all-gather of the codes.  Returns the full code vector."""
+    def reduce_scatter_grad(self, full_grad=None):
+        """Sum the ranks' gradients of the full vector and return this rank's shard of the sum.  Without an
+        argument the gradients are taken from grad_buffer() (no copy); a tensor given here is first copied into
+        that buffer.  Nothing is allocated after the first call."""
+        buf = self.grad_buffer()
+        if full_grad is not None and full_grad.data_ptr() != buf.data_ptr():
+            if full_grad.numel() != self.n_total:
+                raise ValueError("full_grad must have n_total elements")
+            if self.world == 1:
+                return full_grad[self.start: self.end]
+            buf.copy_(full_grad)
+        if self.world == 1:
+            return buf[self.start: self.end]
+        self.dist.reduce_scatter_tensor(self._grad_shard, self._grad_padded, group=self.group)
+        return self._grad_shard[: self.n_own]
+
+    def step(self, grad_shard, wait=True):
+        """One fused step on this rank's shard, then the all-gather of the codes, issued asynchronously (on the
+        collective library's own stream under NCCL) so that whatever the caller enqueues next overlaps it.
+        With wait=True (default) the current stream waits for the gather before this returns the full code vector;
+        with wait=False the caller goes on and `lp` (or wait_gather()) does the waiting when the codes are needed."""
         if grad_shard.numel() != self.n_own:
             raise ValueError("grad_shard must have %d elements" % self.n_own)
+        self.wait_gather()                 # the previous gather must be done before its buffer is rewritten
         self.step_count += 1
         own = self._own_slice()
         if self.n_own:
@@ -104,5 +127,14 @@ class ShardedLowPrecisionAdam:
         if self.world > 1:
             # bytes, so that the collective never meets a dtype it has no name for; in place: this rank's
             # input is its own slice of the output
-            self.dist.all_gather_into_tensor(self.lp_padded.view(torch.uint8), own.view(torch.uint8), group=self.group)
-        return self.lp
+            self._gather = self.dist.all_gather_into_tensor(self.lp_padded.view(torch.uint8), own.view(torch.uint8),
+                                                            group=self.group, async_op=True)
+        if wait:
+            return self.lp
+        return None
+
+    def wait_gather(self):
+        """Make the current stream (the host, on CPU) wait for the pending all-gather, if any."""
+        if self._gather is not None:
+            self._gather.wait()
+            self._gather = None

@@ -93,3 +93,16 @@ def test_format_descriptor_validation(lib):
     for d in bad:
         assert lib.fbsr_format_desc_valid(ctypes.byref(Desc(*d))) == 0, d
     assert lib.fbsr_format_desc_valid(None) == 0
+
+
+def test_python_tile_table_equals_the_library(lib):
+    """The shard grid of the host logic is built from a Python copy of the tile-size rule: it must be the
+    library's for every draw width, and the shard alignment a multiple of each tile size."""
+    import ctypes
+    from paper_2504_20634_b200 import sharding
+    lib.fbsr_tile_elements.argtypes = [ctypes.c_int]
+    lib.fbsr_tile_elements.restype = ctypes.c_size_t
+    for k in range(1, 17):
+        assert sharding.tile_elements(k) == lib.fbsr_tile_elements(k), k
+        assert sharding.SHARD_ALIGN % lib.fbsr_tile_elements(k) == 0
+    assert lib.fbsr_tile_elements(0) == 0 and lib.fbsr_tile_elements(17) == 0

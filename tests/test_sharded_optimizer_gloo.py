@@ -57,9 +57,19 @@ def _worker(rank, world, port, n_total, fmt, out_dir):
         # the unsharded run, on every rank (cheap): one call over the whole vector per step
         w, m, v = w0.numpy().copy(), np.zeros(n_total, np.float32), np.zeros(n_total, np.float32)
         ok = opt.shard_len % sharding.SHARD_ALIGN == 0 and opt.start == min(n_total, rank * opt.shard_len)
+        buffers = set()
         for t in range(steps):
-            shard_grad = opt.reduce_scatter_grad(grads[t][rank])
-            lp = opt.step(shard_grad)
+            if t == 1:
+                # the gradients written straight into the optimizer's persistent buffer, the gather left in flight
+                opt.grad_buffer().copy_(grads[t][rank])
+                shard_grad = opt.reduce_scatter_grad()
+                assert opt.step(shard_grad, wait=False) is None
+                lp = opt.lp
+            else:
+                shard_grad = opt.reduce_scatter_grad(grads[t][rank])
+                lp = opt.step(shard_grad)
+            buffers.add((opt._grad_padded.data_ptr(), opt._grad_shard.data_ptr(), opt.lp_padded.data_ptr()))
+            ok = ok and bool((opt._grad_padded[n_total:] == 0).all())
             acc = grads[t][0].clone()
             for r in range(1, world):
                 acc += grads[t][r]
@@ -67,6 +77,7 @@ def _worker(rank, world, port, n_total, fmt, out_dir):
             got = lp.view(torch.int16).numpy().view(np.uint16) if dt == torch.uint16 else lp.numpy()
             ok = ok and np.array_equal(got, whole)
             ok = ok and np.array_equal(opt.master.numpy(), w[opt.start:opt.end]) and np.array_equal(opt.m.numpy(), m[opt.start:opt.end])
+        ok = ok and len(buffers) == 1          # nothing is reallocated from step to step
         with open(os.path.join(out_dir, "result%d" % rank), "w") as fh:
             fh.write("ok" if ok else "mismatch")
     finally:

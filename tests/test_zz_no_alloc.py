@@ -36,6 +36,17 @@ def _run_pair(fbsr, x, fmt, variant, k, seed, group):
         assert abs(got[key] - ref[key]) <= 1e-9 * max(abs(ref[key]), 1e-3 * ref["sum_abs_e"], 1e-300), key
     assert np.allclose(ge.cpu().numpy(), ref_ge.cpu().numpy(), rtol=1e-9, atol=1e-9)
     assert np.allclose(ge2.cpu().numpy(), ref_ge2.cpu().numpy(), rtol=1e-9, atol=1e-9)
+    # and against the oracle itself, so that this file stands on its own
+    from oracle import capi
+    import gpu_util
+    ecodes, est, ege, _ = capi.fbsr_round_stats(x.cpu().numpy(), fmt, variant, k, seed=seed, offset=3, scale=1.5,
+                                                group_size=group)
+    gpu_util.assert_codes_equal(out, ecodes, "no-alloc codes against the oracle")
+    for key in ("n_finite", "n_up", "n_nan", "n_inf", "n_sat"):
+        assert got[key] == est[key], key
+    for key in ("sum_e", "sum_e2", "sum_signed_e", "sum_abs_e"):
+        assert abs(got[key] - est[key]) <= 1e-9 * max(abs(est[key]), 1e-3 * est["sum_abs_e"], 1e-300), key
+    assert np.allclose(ge.cpu().numpy(), ege, rtol=1e-9, atol=1e-9)
     return got
 
 
@@ -55,6 +66,25 @@ def test_noalloc_statistics_match_the_workspace_entry_point_twice_in_a_row():
     fbsr.fbsr_round_stats_noalloc(x2[:0], torch.empty(0, dtype=torch.uint16, device="cuda"), total, "bf16", "srf", 2, seed=0)
     torch.cuda.synchronize()
     assert all(v == 0 for v in fbsr.stats_from_bytes(total).values())
+
+
+def test_noalloc_call_allocates_nothing():
+    """What the entry point is for: after the first call on the device (which looks up the scratch address),
+    a call neither takes device memory from the driver nor from torch's allocator."""
+    import paper_2504_20634_b200 as fbsr
+    import gpu_util
+    x = torch.from_numpy(gpu_util.mixed_inputs(1_000_003, 903, "e4m3")).cuda()
+    out = torch.empty(x.numel(), dtype=torch.uint8, device="cuda")
+    total = torch.empty(72, dtype=torch.uint8, device="cuda")
+    fbsr.fbsr_round_stats_noalloc(x, out, total, "e4m3", "srf", 3, seed=1)          # warm-up: set-up happens here
+    torch.cuda.synchronize()
+    free0, _ = torch.cuda.mem_get_info()
+    alloc0, reserved0 = torch.cuda.memory_allocated(), torch.cuda.memory_reserved()
+    for seed in (2, 3):
+        fbsr.fbsr_round_stats_noalloc(x, out, total, "e4m3", "srf", 3, seed=seed)
+    torch.cuda.synchronize()
+    assert torch.cuda.mem_get_info()[0] == free0
+    assert (torch.cuda.memory_allocated(), torch.cuda.memory_reserved()) == (alloc0, reserved0)
 
 
 def test_noalloc_rejects_sizes_beyond_its_limit():
