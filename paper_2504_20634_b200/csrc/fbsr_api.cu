@@ -16,6 +16,8 @@ namespace {
 
 typedef int (*dispatch_fn)(const CallArgs&);
 const dispatch_fn kRound[5] = {dispatch_round_0, dispatch_round_1, dispatch_round_2, dispatch_round_3, dispatch_round_4};
+const dispatch_fn kRoundWords[5] = {dispatch_round_words_0, dispatch_round_words_1, dispatch_round_words_2, dispatch_round_words_3, dispatch_round_words_4};
+const dispatch_fn kStats[5] = {dispatch_stats_0, dispatch_stats_1, dispatch_stats_2, dispatch_stats_3, dispatch_stats_4};
 const dispatch_fn kOptim[5] = {dispatch_optim_0, dispatch_optim_1, dispatch_optim_2, dispatch_optim_3, dispatch_optim_4};
 inline bool eight_bit(int fmt) { return fmt == FBSR_E4M3 || fmt == FBSR_E5M2 || fmt == FBSR_B8P4; }
 inline int dispatch_lp(int fmt, const CallArgs& a)
@@ -103,7 +105,7 @@ int fbsr_round_mx(const float* src, void* dst, uint8_t* scales, size_t n, int fm
     CallArgs a = base_args(OP_ROUND_MX, variant, k_bits, n, seed, offset, dst, cuda_stream);
     a.ovf_ieee = ovf_ieee;
     a.src = src; a.scales = scales;
-    return finish(kRound[fmt](a));
+    return finish(kRoundWords[fmt](a));
 }
 
 int fbsr_round_bits(const float* src, void* dst, size_t n, int fmt, int variant, int k_bits,
@@ -117,7 +119,7 @@ int fbsr_round_bits(const float* src, void* dst, size_t n, int fmt, int variant,
     CallArgs a = base_args(OP_ROUND_BITS, variant, k_bits, n, 0, 0, dst, cuda_stream);
     a.ovf_ieee = ovf_ieee;
     a.src = src; a.scale = scale; a.words = rand_words;
-    return finish(kRound[fmt](a));
+    return finish(kRoundWords[fmt](a));
 }
 
 size_t fbsr_stats_workspace_bytes(void) { return (size_t)MAX_SLOW_GRID * sizeof(fbsr_stats); }
@@ -143,7 +145,7 @@ int fbsr_round_stats(const float* src, void* dst, size_t n, int fmt, int variant
             cudaMemsetAsync(group_sum_e2, 0, groups * sizeof(double), a.stream) != cudaSuccess)
             return FBSR_ERR_CUDA;
     }
-    return finish(kRound[fmt](a));
+    return finish(kStats[fmt](a));
 }
 
 }  // extern "C"

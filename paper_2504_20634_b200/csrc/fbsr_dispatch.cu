@@ -1,6 +1,7 @@
 // Kernel instantiations and launch logic for one target format and one group of
-// operations.  Compiled once per (FBSR_FMT, FBSR_GROUP): FBSR_GROUP 0 = rounding
-// entry points, 1 = fused optimizer / accumulation entry points, 2 = 16-bit sources (8-bit targets only).
+// operations.  Compiled once per (FBSR_FMT, FBSR_GROUP): FBSR_GROUP 0 = fbsr_round, 4 = supplied bits and block
+// scales, 5 = rounding with statistics (three units so that they compile in parallel), 1 = fused optimizer and
+// accumulation, 2 = 16-bit sources and the 16-bit-sum update, 3 = the fused Algorithm-1 step (2, 3: 8-bit targets only).
 #include <array>
 #include <utility>
 
@@ -11,7 +12,7 @@
 #error "compile with -DFBSR_FMT=0..4"
 #endif
 #ifndef FBSR_GROUP
-#error "compile with -DFBSR_GROUP=0|1|2|3"
+#error "compile with -DFBSR_GROUP=0..5"
 #endif
 
 namespace fbsr {
@@ -73,7 +74,7 @@ struct Plan { size_t head, n_tiles, tail_begin; bool aligned; };
 template <class Op, bool BITS> struct HasStaged { static constexpr bool value = false; };
 template <> struct HasStaged<RoundOp, false> { static constexpr bool value = true; };
 
-template <class Op, int VAR, int K, bool BITS>
+template <class Op, int VAR, int K, bool BITS, bool IEEE = false>
 int launch_tiles(const Op& op, const CallArgs& a, const Plan& p)
 {
     using T = Tile<K, Op::OCTETS>;
@@ -82,7 +83,7 @@ int launch_tiles(const Op& op, const CallArgs& a, const Plan& p)
     void* dst = static_cast<char*>(a.dst) + p.head * CODE_BYTES;
     const uint64_t call0 = BITS ? 0 : (a.offset + p.head) / T::E;
     const uint32_t* words = BITS ? a.words + p.head / T::DPW : nullptr;
-    if constexpr (HasStaged<Op, BITS>::value) {
+    if constexpr (HasStaged<Op, BITS>::value && !IEEE) {
         if (!p.aligned) {
             const uint64_t want = (p.n_tiles + STAGED_WARPS - 1) / STAGED_WARPS;
             const unsigned grid = (unsigned)(want < 0x7FFFFFF0ull ? want : 0x7FFFFFF0ull) + (tail_count ? 1u : 0u);
@@ -92,7 +93,7 @@ int launch_tiles(const Op& op, const CallArgs& a, const Plan& p)
             return 0;
         }
     }
-    auto kern = tile_kernel<Op, FMT, VAR, K, BITS>;
+    auto kern = tile_kernel<Op, FMT, VAR, K, BITS, IEEE>;
     // One tile per warp, CTAs handed out by the hardware scheduler.  A persistent grid with a static
     // tile stride measured 5-10 % slower here: multiprocessors do not all see the same memory
     // bandwidth, and a static split makes the whole launch wait for the slowest of them.
@@ -143,55 +144,24 @@ Plan make_plan(const Op& op, const CallArgs& a)
     return p;
 }
 
-// The IEEE reading of overflow after a saturating pass: only finite values beyond M differ (M + ulp/2 and above
-// become the infinity, or the NaN of a format without one), and they need no draw.  For ops whose value can be
-// formed again from their inputs (plain rounding and 16-bit sources) the call runs the tiled kernels as usual and
-// this kernel then rewrites those elements, one element per thread; the other ops use the general kernel.
-template <class Op> struct Restartable { static constexpr bool value = false; };
-template <> struct Restartable<RoundOp> { static constexpr bool value = true; };
-template <int SRC> struct Restartable<LpSrcOp<SRC>> { static constexpr bool value = true; };
-
-template <class Op>
-__global__ void __launch_bounds__(CTA_THREADS)
-overflow_fixup_kernel(const Op op, void* __restrict__ dst, const uint64_t n)
-{
-    // a CTA takes chunks of 8 x 256 elements; a thread's 8 loads are independent and coalesced across the warp
-    constexpr int PER_THREAD = 8;
-    constexpr uint64_t CHUNK = (uint64_t)PER_THREAD * CTA_THREADS;
-    for (uint64_t base = (uint64_t)blockIdx.x * CHUNK; base < n; base += (uint64_t)gridDim.x * CHUNK) {
-        uint32_t bits[PER_THREAD];
-#pragma unroll
-        for (int j = 0; j < PER_THREAD; ++j) {
-            const uint64_t i = base + (uint64_t)j * CTA_THREADS + threadIdx.x;
-            bits[j] = i < n ? op.scalar(i) : 0u;
-        }
-#pragma unroll
-        for (int j = 0; j < PER_THREAD; ++j) {
-            const uint64_t i = base + (uint64_t)j * CTA_THREADS + threadIdx.x;
-            const uint32_t mag = bits[j] & 0x7FFFFFFFu;
-            if (mag > Format<FMT>::MAXBITS && mag < 0x7F800000u)
-                store_code1<FMT>(dst, i, round_core<FMT, false>(bits[j], 0u, RTNE, 1, nullptr, true));
-        }
-    }
-}
+// The IEEE reading of overflow (finite values beyond M) is a template variant of the tiled kernel for the ops
+// listed here (plain rounding with generated draws, 16-bit sources); the other calls use the general kernel.
+template <class Op, bool BITS> struct HasIeee { static constexpr bool value = false; };
+template <> struct HasIeee<RoundOp, false> { static constexpr bool value = true; };
+template <int SRC> struct HasIeee<LpSrcOp<SRC>, false> { static constexpr bool value = true; };
 
 template <class Op, int VAR, int K, bool BITS>
 int run(const Op& op, const CallArgs& a)
 {
-    const Plan p = make_plan<Op, K, BITS>(op, a);
-    const bool fixup = a.ovf_ieee && Restartable<Op>::value;
-    if (p.n_tiles == 0 || (a.ovf_ieee && !fixup)) return launch_generic<Op, BITS, false>(op, a, 0, a.n, nullptr);
-    CallArgs sat = a;
-    sat.ovf_ieee = 0;                                  // the head, too, saturates first when the fix-up pass follows
-    launch_generic<Op, BITS, false>(op, sat, 0, p.head, nullptr);
-    launch_tiles<Op, VAR, K, BITS>(op, a, p);          // whole tiles and the ragged end
-    if (fixup) {
-        const uint64_t want = ((uint64_t)a.n + 8 * CTA_THREADS - 1) / (8 * CTA_THREADS);
-        const unsigned grid = (unsigned)(want < (uint64_t)MAX_SLOW_GRID ? want : (uint64_t)MAX_SLOW_GRID);   // resident CTAs loop over the chunks
-        overflow_fixup_kernel<Op><<<grid, CTA_THREADS, 0, a.stream>>>(op, a.dst, (uint64_t)a.n);
-        count_launch();
+    Plan p = make_plan<Op, K, BITS>(op, a);
+    constexpr bool ieee_tiles = HasIeee<Op, BITS>::value;
+    if (a.ovf_ieee && !(ieee_tiles && p.aligned)) p.n_tiles = 0;
+    if (p.n_tiles == 0) return launch_generic<Op, BITS, false>(op, a, 0, a.n, nullptr);
+    launch_generic<Op, BITS, false>(op, a, 0, p.head, nullptr);
+    if constexpr (ieee_tiles) {
+        if (a.ovf_ieee) return launch_tiles<Op, VAR, K, BITS, true>(op, a, p);
     }
-    return 0;
+    return launch_tiles<Op, VAR, K, BITS>(op, a, p);          // whole tiles and the ragged end
 }
 
 // ---- (variant, k) -> instantiation
@@ -221,7 +191,7 @@ int by_variant_and_k(const Op& op, const CallArgs& a)
 #define FBSR_CAT_(a, b) a##b
 #define FBSR_CAT(a, b) FBSR_CAT_(a, b)
 
-#if FBSR_GROUP == 0
+#if FBSR_GROUP == 5
 namespace {
 // Statistics: the head of the call (up to the first tile boundary of the draw stream) and the ragged end go to the
 // general kernel, whole tiles to the tiled statistics kernel; every CTA leaves one partial in the workspace (tiles
@@ -296,14 +266,18 @@ int stats_by_variant_and_k(const CallArgs& a)
 }
 }  // namespace
 
+int FBSR_CAT(dispatch_stats_, FBSR_FMT)(const CallArgs& a) { return stats_by_variant_and_k(a); }
+#elif FBSR_GROUP == 0
 int FBSR_CAT(dispatch_round_, FBSR_FMT)(const CallArgs& a)
 {
-    const RoundOp op{a.src, a.scale};
+    return by_variant_and_k<RoundOp, false>(RoundOp{a.src, a.scale}, a);
+}
+#elif FBSR_GROUP == 4
+int FBSR_CAT(dispatch_round_words_, FBSR_FMT)(const CallArgs& a)
+{
     switch (a.op) {
-    case OP_ROUND: return by_variant_and_k<RoundOp, false>(op, a);
-    case OP_ROUND_BITS: return by_variant_and_k<RoundOp, true>(op, a);
+    case OP_ROUND_BITS: return by_variant_and_k<RoundOp, true>(RoundOp{a.src, a.scale}, a);
     case OP_ROUND_MX: return by_variant_and_k<MxOp<FMT>, false>(MxOp<FMT>{a.src, a.scales, a.n}, a);
-    case OP_ROUND_STATS: return stats_by_variant_and_k(a);
     default: return 1;
     }
 }

@@ -43,6 +43,8 @@ constexpr int MAX_SLOW_GRID = 148 * 8;      // CTAs of the general kernel; also 
 // (dispatch_lp_* and dispatch_qat_adamw_* exist for the 8-bit targets only).
 #define FBSR_DECLARE_DISPATCH(fmt) \
     int dispatch_round_##fmt(const CallArgs&); \
+    int dispatch_round_words_##fmt(const CallArgs&); \
+    int dispatch_stats_##fmt(const CallArgs&); \
     int dispatch_optim_##fmt(const CallArgs&);\
     int dispatch_lp_##fmt(const CallArgs&); \
     int dispatch_qat_adamw_##fmt(const CallArgs&);

@@ -618,7 +618,24 @@ __device__ __forceinline__ void pack_row_fast(const uint32_t (&t)[8], const floa
 // tile per warp; the loop only matters when the grid had to be capped.
 // call0: global index of the Philox call that serves element 0 (Philox source), or
 // words: the packed word stream whose word 0 serves element 0 (supplied bits).
-template <class Op, int FMT, int VAR, int K, bool BITS>
+// IEEE: finite values beyond M are rounded as IEEE nearest-even does (Section II read literally) instead of
+// saturating: M below the midpoint to the next power of two, the infinity (the NaN code of a format without one)
+// from there on, the midpoint itself to whichever of the two has an even code.  The row rounder has already
+// clamped such an element to the code of M, so one comparison and one select per element put the other code in
+// place; bfloat16 rows holding such a value are redone element by element anyway.
+template <int FMT> struct IeeeOverflow {
+    using F = Format<FMT>;
+    static constexpr uint32_t TIE_BITS = F::MAXBITS + (1u << (24 - F::P - 1));      // M + ulp(M) / 2, exact in binary32
+    static constexpr bool TIE_OVERFLOWS = (F::MAXCODE & 1u) != 0;                   // the code of M is odd: the tie leaves it
+    static constexpr uint32_t CODE = F::HAS_INF ? F::INFCODE : F::NANCODE;
+    __device__ __forceinline__ static bool beyond(float y)
+    {
+        const float tie = __uint_as_float(TIE_BITS);
+        return TIE_OVERFLOWS ? fabsf(y) >= tie : fabsf(y) > tie;
+    }
+};
+
+template <class Op, int FMT, int VAR, int K, bool BITS, bool IEEE = false>
 __global__ void __launch_bounds__(CTA_THREADS, Op::MIN_CTAS)
 tile_kernel(const Op op, void* __restrict__ dst, const uint64_t n_tiles, const uint64_t call0,
             const uint32_t k0, const uint32_t k1, const uint32_t* __restrict__ words, const uint32_t tail_count)
@@ -643,7 +660,7 @@ tile_kernel(const Op op, void* __restrict__ dst, const uint64_t n_tiles, const u
                 word = ws == 0 ? o.x : ws == 1 ? o.y : ws == 2 ? o.z : o.w;
             }
             const uint32_t n = (word >> ((j % T::DPW) * K)) & T::MASK;
-            store_code1<FMT>(dst, p, round_core<FMT, false>(op.scalar(p), n, VAR, K, nullptr));
+            store_code1<FMT>(dst, p, round_core<FMT, false>(op.scalar(p), n, VAR, K, nullptr, IEEE));
         }
         return;
     }
@@ -718,6 +735,11 @@ tile_kernel(const Op op, void* __restrict__ dst, const uint64_t n_tiles, const u
                         }
                         uint32_t t[8];
                         const bool redo = round_row_fast<FMT, VAR, K>(y, d, t);
+                        if constexpr (IEEE && FMT != BF16) {
+#pragma unroll
+                            for (int i = 0; i < 8; ++i)
+                                t[i] = IeeeOverflow<FMT>::beyond(y[i]) ? IeeeOverflow<FMT>::CODE << (32 - Format<FMT>::K) : t[i];
+                        }
                         if (!redo) {
                             pack_row_fast<FMT>(t, y, packed + o * WPO);
                         } else {
@@ -728,7 +750,7 @@ tile_kernel(const Op op, void* __restrict__ dst, const uint64_t n_tiles, const u
                                 uint32_t bits;
                                 if constexpr (OCT == 1) bits = op.exact_bits(regs[j], i, y[i]);
                                 else bits = op.exact_bits(regs[j], o, i, y[i]);
-                                c[i] = round_core<FMT, false>(bits, d.template at<0>(i), VAR, K, nullptr);
+                                c[i] = round_core<FMT, false>(bits, d.template at<0>(i), VAR, K, nullptr, IEEE);
                             }
                             pack_codes8<FMT>(c, packed + o * WPO);
                         }

@@ -35,13 +35,14 @@ def main():
     dev = torch.device("cuda", 0)
     scale = args.scale
     if args.data == "fp8act":
-        x, scale = workloads.fp8_activations(args.fmt, rows=n // 32768, cols=32768, device=dev)
+        x, scale = workloads.fp8_activations(base_fmt, rows=n // 32768, cols=32768, device=dev)
     elif args.misalign:
         x = workloads.bandwidth_sweep(n + args.misalign, seed=1234, device=dev)[args.misalign:]
     else:
         x = workloads.bandwidth_sweep(n, seed=1234, device=dev)
-    code_bytes = 2 if args.fmt in ("bf16", "fp16") else 1
-    out = torch.empty(n, dtype=fbsr.CODE_DTYPE[args.fmt], device=dev)
+    base_fmt = args.fmt.split("+")[0]               # "fp16+ieee": the IEEE overflow option
+    code_bytes = 2 if base_fmt in ("bf16", "fp16") else 1
+    out = torch.empty(n, dtype=fbsr.CODE_DTYPE[base_fmt], device=dev)
     if args.op == "round":
         bytes_per_elem = 4 + code_bytes
         run = lambda s: fbsr.fbsr_round(x, args.fmt, args.variant, args.k, seed=1234, scale=scale, out=out)
