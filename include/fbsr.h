@@ -37,7 +37,11 @@
  *   - Any n (including 0) and any element alignment are accepted.  The fast
  *     path needs src 32-byte aligned, dst 16-byte aligned and `offset` a multiple
  *     of the tile size reported by fbsr_tile_elements(); other calls are served
- *     by a slower kernel with identical results.
+ *     by a slower kernel with identical results.  fbsr_round itself has a second
+ *     fast kernel that takes pointers of any element alignment (a slice of a
+ *     tensor, a packed parameter buffer) at about four fifths of the speed; the
+ *     part of a call before the first tile boundary of `offset` (less than one
+ *     tile) always goes to the slower kernel.
  *   - Errors are reported by the return value only.  Nothing is written on error.
  */
 #ifndef FBSR_H
@@ -70,11 +74,11 @@ typedef enum {
                       0x7F / 0xFF are +-Inf, 0x80 is the NaN, there is no negative zero */
 } fbsr_fmt;
 
-/* May be or-ed into any `fmt` argument.  Section II says that values beyond the finite range are "rounded
- * deterministically as in IEEE-754 round to nearest"; with this flag finite |y| > M follow that reading
- * (M below M + ulp(M)/2, +-Inf above it -- the NaN code for e4m3 -- ties to the even neighbour) instead
- * of saturating.  fbsr_round, fbsr_round_bits and fbsr_round_lp serve the flag with a second pass over the input
- * that rewrites the values beyond M (about a third of the usual speed); the other calls use the general kernel. */
+/* May be or-ed into any `fmt` argument.  Section II leaves values beyond the finite range to the deterministic
+ * nearest rounding of IEEE 754; with this flag finite |y| > M follow that reading (M below M + ulp(M)/2, +-Inf
+ * above it -- the NaN code for e4m3 -- ties to the even neighbour) instead of saturating.  fbsr_round and
+ * fbsr_round_lp serve the flag at full speed on aligned calls (one comparison per element in the tiled kernel);
+ * the other entry points, and calls whose pointers are off the fast path's alignment, use the general kernel. */
 #define FBSR_OVF_IEEE 0x100
 
 /* Round-up predicates: the few-bit stochastic ones of Section II-B and Eq. (8), and the deterministic
@@ -113,18 +117,19 @@ typedef struct {
 int fbsr_round(const float* src, void* dst, size_t n, int fmt, int variant, int k_bits,
                uint64_t seed, uint64_t offset, float scale, void* cuda_stream);
 
-/* fbsr_round_lp -- the paper's own regime (Section III-E, Fig. 2, Algorithm 1 "w8 <- RoundTo8(...)"):
+/* fbsr_round_lp -- the paper's own regime (Section III-E, Fig. 2, the rounding to 8 bits that ends Algorithm 1):
  * the source is already a low-precision tensor.  dst[i] = FBSR(fl32(value(src[i]) * scale)), where
  * value() widens the stored code exactly by Eq. (1).
  *   src      device, n codes of src_fmt (FBSR_BF16 or FBSR_FP16, uint16 each); must not overlap dst
  *   dst      device, n codes of dst_fmt (FBSR_E4M3, FBSR_E5M2 or FBSR_B8P4, uint8 each)
- * Other format pairs return FBSR_ERR_UNSUPPORTED.  The fast path needs src and dst 16-byte aligned
- * (8-byte for dst) and `offset` on the tile grid, like fbsr_round.  A NaN source keeps its sign. */
+ * Other format pairs return FBSR_ERR_UNSUPPORTED.  The fast path needs src 32-byte aligned, dst 16-byte
+ * aligned (a lane reads 16 source codes and writes 16 target codes at a time) and `offset` on the tile grid;
+ * other calls are served by the general kernel with identical results.  A NaN source keeps its sign. */
 int fbsr_round_lp(const void* src, int src_fmt, void* dst, size_t n, int dst_fmt, int variant, int k_bits,
                   uint64_t seed, uint64_t offset, float scale, void* cuda_stream);
 
 /* fbsr_round_desc -- fbsr_round for a format (K, P, B; M) given at run time, Section II's parametrisation
- * ("a binary floating-point format is described by the tuple (K, P, B; M)"); the rounding itself is Section II-A
+ * (width, precision, exponent bias and largest finite value); the rounding itself is Section II-A
  * Eq. (2)-(5) with the predicates of Section II-B and Eq. (8), as in fbsr_round.
  *   desc     HOST pointer, read before the call returns:
  *     K          8 or 16: width of a code (dst is uint8 or uint16)
@@ -157,8 +162,8 @@ int fbsr_round_desc(const float* src, void* dst, size_t n, const fbsr_format_des
 /* 1 if fbsr_round_desc accepts the descriptor, else 0.  Host only, no CUDA call. */
 int fbsr_format_desc_valid(const fbsr_format_desc* desc);
 
-/* fbsr_round_mx -- block-scaled tensors (Section I-A: "blocks of low-precision values are accompanied by a
- * scale factor, which may be a power of two").  Blocks are 32 consecutive elements of the call; per block
+/* fbsr_round_mx -- block-scaled tensors (Section I-A: each block of low-precision values carries a scale
+ * factor of its own, here a power of two).  Blocks are 32 consecutive elements of the call; per block
  *     amax  = largest finite |src| (0 if none)
  *     e_blk = clamp(floor(log2 amax) - emax, -127, 127), emax = floor(log2 M);  -127 if amax < 2^-126
  *     scales[block] = e_blk + 127;   dst[i] = FBSR(fl32(src[i] * 2^-e_blk))
@@ -170,8 +175,8 @@ int fbsr_round_mx(const float* src, void* dst, uint8_t* scales, size_t n, int fm
                   uint64_t seed, uint64_t offset, void* cuda_stream);
 
 /* fbsr_round_bits -- the same rounding with caller-supplied random bits
- * (Section II-B: "random numbers will be supplied as a finite sequence of random
- * bits").  rand_words: device, ceil(n / dpw) words; element i uses field
+ * (Section II-B treats the randomness as a finite string of bits handed to the
+ * rounder).  rand_words: device, ceil(n / dpw) words; element i uses field
  * (i mod dpw) of word (i / dpw), low bits first; higher bits are ignored. */
 int fbsr_round_bits(const float* src, void* dst, size_t n, int fmt, int variant, int k_bits,
                     const uint32_t* rand_words, float scale, void* cuda_stream);
@@ -215,7 +220,9 @@ int fbsr_round_stats(const float* src, void* dst, size_t n, int fmt, int variant
  *     occupy the shared scratch.
  *   - The first call on each device looks up the device address of the scratch
  *     array (cudaGetSymbolAddress) with that device current; make that first
- *     call outside any stream capture.
+ *     call outside any stream capture.  The address is remembered per device
+ *     ordinal for the life of the process and does not survive a
+ *     cudaDeviceReset: do not call this entry point again after one.
  *   - All calls on a device share the one array.  It keeps whatever the previous
  *     call left there; nothing in it has to start at zero, because every slot a
  *     call reads is first written by that same call.  Two calls that can overlap
@@ -248,7 +255,14 @@ int fbsr_adam_update(float* master_w, const float* grad, float* m, float* v, voi
                      int fmt, int variant, int k_bits, uint64_t seed, uint64_t offset,
                      float lr, float beta1, float beta2, float eps, int step, void* cuda_stream);
 
-/* fbsr_accumulate -- Algorithm 1, "w8 <- RoundTo8(w16 + u16)" with the sum
+/* The four host scalars of fbsr_adam_update and fbsr_qat_adamw_step for a given step (Algorithm 1 leaves the
+ * arithmetic of its AdamW update open; this is the library's definition, stated with fbsr_adam_update):
+ * out = {c1, c2, a1, a2}.  beta^step is formed by repeated multiplication in binary64; the multiplication stops
+ * once the product of a |beta| < 1 has fallen below 2^-54, from where on 1 - beta^step is exactly 1, so the cost
+ * on the host does not grow with the step count.  Host only, no CUDA call; out must hold 4 floats. */
+void fbsr_adam_scalars(float lr, float beta1, float beta2, int step, float out[4]);
+
+/* fbsr_accumulate -- the last step of Algorithm 1 (weight plus update, rounded to the narrow format) with the sum
  * formed in binary32:  w_lp[i] = FBSR(fl32(value(w_lp[i]) + update[i])), in place.
  * A NaN sum is written as the positive quiet NaN. */
 int fbsr_accumulate(void* w_lp, const float* update, size_t n, int fmt, int variant, int k_bits,
@@ -256,12 +270,12 @@ int fbsr_accumulate(void* w_lp, const float* update, size_t n, int fmt, int vari
 
 /* fbsr_qat_adamw_step -- Algorithm 1, one whole iteration from the gradient on, fused:
  *     w16 = value(w8);  g = value(grad16);
- *     "AdamW update in F16": moments in binary32, each operation rounded once, the result rounded to the 16-bit format
+ *     the algorithm's 16-bit AdamW update: moments in binary32, each operation rounded once, the result rounded to the 16-bit format
  *         m' = fma(beta1, m, a1 g);  v' = fma(beta2, v, (a2 g) g);  d = sqrt(v') c2 + eps;
  *         u32 = fma(-c1, m' / d, -(lr weight_decay) w16);   u16 = RTNE_16(u32)      (c1, c2, a1, a2 as in fbsr_adam_update)
  *     w8 = FBSR(RTNE_16(fl32(w16 + u16)))                                            (as in fbsr_qat_update; SR applied here)
  *   w8       device, n codes of w_fmt (FBSR_E4M3, FBSR_E5M2 or FBSR_B8P4), read and overwritten
- *   grad16   device, n codes of g_fmt (FBSR_BF16 or FBSR_FP16), the "F16" of the algorithm
+ *   grad16   device, n codes of g_fmt (FBSR_BF16 or FBSR_FP16), the algorithm's 16-bit format
  *   m, v     device, n binary32 moments each, read and overwritten
  * 20 bytes per parameter.  The paper states the shape of the step, not its arithmetic: the operation list is this
  * library's.  A NaN result is written as the positive NaN code; m and v then hold NaNs of unspecified sign. */
@@ -280,9 +294,13 @@ int fbsr_qat_update(void* w8, const void* update16, size_t n, int w_fmt, int u_f
 /* fbsr_round_host -- fbsr_round for HOST buffers (pinned memory gives overlap):
  * copies src to the device in chunks, rounds, copies the codes back, using
  * dev_workspace (device, >= fbsr_round_host_min_workspace() bytes, 256-byte
- * aligned) as a double buffer.  Work is enqueued on cuda_stream and on an
- * internal copy stream that is joined back into cuda_stream before return;
- * dst_host is valid once cuda_stream has been synchronised. */
+ * aligned) as a double buffer.  Kernels are enqueued on cuda_stream, the copies
+ * on two internal streams (one per direction, so that the upload of a chunk, the
+ * rounding of the previous one and the download of the one before overlap); the
+ * uploads wait for what cuda_stream held at the time of the call, and everything
+ * is joined back into cuda_stream before return: dst_host is valid once
+ * cuda_stream has been synchronised.  Callers on different streams may call
+ * concurrently with workspaces of their own. */
 size_t fbsr_round_host_min_workspace(void);
 int fbsr_round_host(const float* src_host, void* dst_host, size_t n, int fmt, int variant, int k_bits,
                     uint64_t seed, uint64_t offset, float scale, void* dev_workspace,

@@ -245,8 +245,8 @@ done:
 uint32_t fbsr_oracle_round_one(float y, int fmt, int variant, int N, uint32_t n,
                                int* kind_out, int* up_out, double* delta_out)
 {
-    /* bit 8 of fmt selects the paper-literal treatment of finite values beyond M (Section II: "rounded
-       deterministically as in IEEE-754 round to nearest"): below M + ulp(M)/2 they give M, from there on
+    /* bit 8 of fmt selects the paper-literal treatment of finite values beyond M (Section II hands them to the
+       deterministic nearest rounding of IEEE 754): below M + ulp(M)/2 they give M, from there on
        the infinity (the NaN code where the format has no infinity).  Without it they saturate to M. */
     return round_one_f(y, &FORMATS[fmt & 0xFF], (fmt >> 8) & 1, variant, N, n, kind_out, up_out, delta_out);
 }
@@ -316,8 +316,8 @@ int fbsr_oracle_round_lp(const void* src, int src_fmt, void* dst, size_t n, int 
     return 0;
 }
 
-/* Block-scaled tensors (Section I-A: "blocks of low-precision values are accompanied by a scale factor,
- * which may be a power of two").  Blocks are 32 consecutive elements of the call.  Per block:
+/* Block-scaled tensors (Section I-A: every block of low-precision values carries its own scale factor, here
+ * a power of two).  Blocks are 32 consecutive elements of the call.  Per block:
  *   amax = largest finite |x| (0 if none);  e_blk = clamp(floor(log2 amax) - emax, -127, 127) with
  *   emax = floor(log2 M) of the target and e_blk = -127 for amax = 0 or subnormal;
  *   scale byte = e_blk + 127;  y = fl32(x 2^-e_blk);  code = FBSR(y).
@@ -448,8 +448,8 @@ int fbsr_oracle_adam_update(float* w, const float* g, float* m, float* v, void* 
     return 0;
 }
 
-/* Algorithm 1, last line, with the sum formed in the 16-bit format as the algorithm states
- * ("w8 <- RoundTo8(w16 + u16)"): w16 = value(w8) exactly; s = fl32(w16 + u16) rounded to the 16-bit
+/* Algorithm 1, last line (the 8-bit weight rounded from the 16-bit sum of weight and update), with the sum
+ * formed in the 16-bit format as the algorithm states: w16 = value(w8) exactly; s = fl32(w16 + u16) rounded to the 16-bit
  * format with ties to even (saturating like every other rounding here); w8' = FBSR(s).  Forming the
  * 16-bit sum by way of one binary32 addition is this library's definition. */
 int fbsr_oracle_qat_update(void* w8, const void* u16, size_t n, int w_fmt, int u_fmt, int variant, int k,
@@ -470,7 +470,7 @@ int fbsr_oracle_qat_update(void* w8, const void* u16, size_t n, int w_fmt, int u
 
 /* Algorithm 1, one whole iteration per parameter, from the gradient on:
  *   w16 = value(w8)  (exact);  g = value(g16);
- *   "AdamW update in F16": moments in binary32, every operation rounded once, the result rounded to F16:
+ *   the algorithm's 16-bit AdamW update: moments in binary32, every operation rounded once, the result rounded to F16:
  *     m' = fma(b1, m, a1 g);  v' = fma(b2, v, (a2 g) g);  d = sqrt(v') c2 + eps;
  *     u32 = fma(-c1, m'/d, -(lr wd) w16);   u16 = RTNE_F16(u32)          (c1, c2, a1, a2 as for Adam)
  *   w8' = FBSR(RTNE_F16(fl32(w16 + u16)))                                 (the step above)

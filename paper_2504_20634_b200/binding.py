@@ -77,6 +77,8 @@ def _load():
     L.fbsr_round_host_min_workspace.argtypes = []
     L.fbsr_round_host_min_workspace.restype = sz
     L.fbsr_round_host.argtypes = [vp, vp, sz, i, i, i, u64, u64, f, vp, sz, vp]
+    L.fbsr_adam_scalars.argtypes = [f, f, f, i, ctypes.POINTER(ctypes.c_float)]
+    L.fbsr_adam_scalars.restype = None
     L.fbsr_tile_elements.argtypes = [i]
     L.fbsr_tile_elements.restype = sz
     L.fbsr_launch_count.argtypes = []
@@ -108,6 +110,13 @@ def fbsr_version():
 
 def fbsr_tile_elements(k_bits):
     return int(_L.fbsr_tile_elements(int(k_bits)))
+
+
+def fbsr_adam_scalars(lr, beta1, beta2, step):
+    """(c1, c2, a1, a2) of fbsr_adam_update / fbsr_qat_adamw_step as binary32 values (host only)."""
+    out = (ctypes.c_float * 4)()
+    _L.fbsr_adam_scalars(lr, beta1, beta2, step, out)
+    return tuple(float(x) for x in out)
 
 
 def fbsr_launch_count():

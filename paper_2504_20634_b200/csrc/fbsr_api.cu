@@ -50,6 +50,32 @@ CallArgs base_args(OpKind op, int variant, int k, size_t n, uint64_t seed, uint6
     return a;
 }
 
+// beta^step by repeated multiplication in binary64 (the definition shared with the oracle).  Once the running
+// product of a |beta| < 1 is below 2^-54 it no longer matters: 1 - product rounds to exactly 1.0, so the loop
+// stops there and a long run does not pay for its step count on the host.
+double beta_power(float beta, int step)
+{
+    const double b = (double)beta;
+    const bool shrinking = std::fabs(b) < 1.0;
+    double p = 1.0;
+    for (int t = 0; t < step; ++t) {
+        p *= b;
+        if (shrinking && std::fabs(p) < 0x1p-54) break;
+    }
+    return p;
+}
+
+// Host scalars of the Adam steps: out = {lr / (1 - beta1^step), 1 / sqrt(1 - beta2^step), 1 - beta1, 1 - beta2},
+// each formed in binary64 and rounded once to binary32.
+void adam_scalars(float lr, float beta1, float beta2, int step, float out[4])
+{
+    const double b1t = beta_power(beta1, step), b2t = beta_power(beta2, step);
+    out[0] = (float)((double)lr / (1.0 - b1t));
+    out[1] = (float)(1.0 / std::sqrt(1.0 - b2t));
+    out[2] = (float)(1.0 - (double)beta1);
+    out[3] = (float)(1.0 - (double)beta2);
+}
+
 int check_round(const float* src, const void* dst, size_t n, int fmt, int variant, int k, float scale)
 {
     if (bad_enum(fmt, variant, k)) return FBSR_ERR_INVALID_ARG;
@@ -215,17 +241,13 @@ int fbsr_adam_update(float* master_w, const float* grad, float* m, float* v, voi
     if (misaligned(master_w, 4) || misaligned(grad, 4) || misaligned(m, 4) || misaligned(v, 4) ||
         misaligned(dst_lp, code_bytes(fmt))) return FBSR_ERR_ALIGNMENT;
     if (n == 0) return FBSR_OK;
-    // Bias-correction scalars in binary64, rounded once to binary32.
-    double b1t = 1.0, b2t = 1.0;
-    for (int t = 0; t < step; ++t) { b1t *= (double)beta1; b2t *= (double)beta2; }
+    float sc[4];
+    adam_scalars(lr, beta1, beta2, step, sc);
     CallArgs a = base_args(OP_ADAM, variant, k_bits, n, seed, offset, dst_lp, cuda_stream);
     a.ovf_ieee = ovf_ieee;
     a.w = master_w; a.g = grad; a.m = m; a.v = v;
     a.beta1 = beta1; a.beta2 = beta2; a.eps = eps;
-    a.neg_c1 = -(float)((double)lr / (1.0 - b1t));
-    a.c2 = (float)(1.0 / std::sqrt(1.0 - b2t));
-    a.a1 = (float)(1.0 - (double)beta1);
-    a.a2 = (float)(1.0 - (double)beta2);
+    a.neg_c1 = -sc[0]; a.c2 = sc[1]; a.a1 = sc[2]; a.a2 = sc[3];
     return finish(kOptim[fmt](a));
 }
 
@@ -268,20 +290,23 @@ int fbsr_qat_adamw_step(void* w8, const void* grad16, float* m, float* v, size_t
     if (n > 0 && (!w8 || !grad16 || !m || !v)) return FBSR_ERR_INVALID_ARG;
     if (misaligned(grad16, 2) || misaligned(m, 4) || misaligned(v, 4)) return FBSR_ERR_ALIGNMENT;
     if (n == 0) return FBSR_OK;
-    double b1t = 1.0, b2t = 1.0;
-    for (int t = 0; t < step; ++t) { b1t *= (double)beta1; b2t *= (double)beta2; }
+    float sc[4];
+    adam_scalars(lr, beta1, beta2, step, sc);
     CallArgs a = base_args(OP_QAT_ADAMW, variant, k_bits, n, seed, offset, w8, cuda_stream);
     a.ovf_ieee = ovf_ieee;
     a.src_lp = grad16; a.src_fmt = g_fmt; a.m = m; a.v = v;
     a.beta1 = beta1; a.beta2 = beta2; a.eps = eps;
-    a.neg_c1 = -(float)((double)lr / (1.0 - b1t));
-    a.c2 = (float)(1.0 / std::sqrt(1.0 - b2t));
-    a.a1 = (float)(1.0 - (double)beta1);
-    a.a2 = (float)(1.0 - (double)beta2);
+    a.neg_c1 = -sc[0]; a.c2 = sc[1]; a.a1 = sc[2]; a.a2 = sc[3];
     const volatile float lrwd = lr * weight_decay;           // one rounded binary32 product
     a.neg_lrwd = -lrwd;
     return finish(w_fmt == FBSR_E4M3 ? dispatch_qat_adamw_2(a) : w_fmt == FBSR_E5M2 ? dispatch_qat_adamw_3(a)
                                                                                    : dispatch_qat_adamw_4(a));
+}
+
+void fbsr_adam_scalars(float lr, float beta1, float beta2, int step, float out[4])
+{
+    if (out == nullptr) return;
+    adam_scalars(lr, beta1, beta2, step < 1 ? 1 : step, out);
 }
 
 size_t fbsr_tile_elements(int k_bits)
@@ -305,22 +330,33 @@ int fbsr_round_host(const float* src_host, void* dst_host, size_t n, int fmt, in
     if (misaligned(dev_workspace, 256)) return FBSR_ERR_ALIGNMENT;
     if (n == 0) return FBSR_OK;
 
-    // Per-device copy stream and events, created on first use and kept for the life of the process.
-    struct Side { cudaStream_t d2h = nullptr; cudaEvent_t rounded[2] = {nullptr, nullptr}, drained[2] = {nullptr, nullptr}; bool ok = false; };
+    // Per-device copy streams (one per direction), created on first use and kept for the life of the process;
+    // the lock covers only that creation.  The events are made per call, so concurrent callers on different
+    // streams share nothing but the two copy streams, in which their copies simply queue.
+    struct Side { cudaStream_t h2d = nullptr, d2h = nullptr; bool ok = false; };
     static Side sides[64];
     static std::mutex mu;
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return FBSR_ERR_CUDA;
-    std::lock_guard<std::mutex> lock(mu);
-    Side& s = sides[dev];
-    if (!s.ok) {
-        if (cudaStreamCreateWithFlags(&s.d2h, cudaStreamNonBlocking) != cudaSuccess) return FBSR_ERR_CUDA;
-        for (int i = 0; i < 2; ++i) {
-            if (cudaEventCreateWithFlags(&s.rounded[i], cudaEventDisableTiming) != cudaSuccess ||
-                cudaEventCreateWithFlags(&s.drained[i], cudaEventDisableTiming) != cudaSuccess) return FBSR_ERR_CUDA;
+    Side s;
+    {
+        std::lock_guard<std::mutex> lock(mu);
+        Side& shared = sides[dev];
+        if (!shared.ok) {
+            if (cudaStreamCreateWithFlags(&shared.h2d, cudaStreamNonBlocking) != cudaSuccess ||
+                cudaStreamCreateWithFlags(&shared.d2h, cudaStreamNonBlocking) != cudaSuccess) return FBSR_ERR_CUDA;
+            shared.ok = true;
         }
-        s.ok = true;
+        s = shared;
     }
+    // uploaded / rounded / drained per slot, and the fork point of the caller's stream
+    struct Events {
+        cudaEvent_t e[7] = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
+        bool create() { for (auto& x : e) if (cudaEventCreateWithFlags(&x, cudaEventDisableTiming) != cudaSuccess) return false; return true; }
+        ~Events() { for (auto x : e) if (x) cudaEventDestroy(x); }      // released by the runtime once the work has run
+    } ev;
+    if (!ev.create()) return FBSR_ERR_CUDA;
+    cudaEvent_t* uploaded = ev.e; cudaEvent_t* rounded = ev.e + 2; cudaEvent_t* drained = ev.e + 4; cudaEvent_t start = ev.e[6];
 
     const cudaStream_t main = static_cast<cudaStream_t>(cuda_stream);
     const size_t cb = code_bytes(fmt);
@@ -348,27 +384,34 @@ int fbsr_round_host(const float* src_host, void* dst_host, size_t n, int fmt, in
     }
     if (2 * (in_bytes + out_bytes) > workspace_bytes) return FBSR_ERR_WORKSPACE;
 
+    // the uploads start after whatever the caller's stream held at the time of the call
+    if (cudaEventRecord(start, main) != cudaSuccess || cudaStreamWaitEvent(s.h2d, start, 0) != cudaSuccess) return FBSR_ERR_CUDA;
     bool used[2] = {false, false};
     size_t idx = 0;
     for (size_t at = 0; at < n; at += chunk, ++idx) {
         const int sl = (int)(idx & 1);
         const size_t len = n - at < chunk ? n - at : chunk;
-        // the slot's previous codes must have left before its buffers are reused
-        if (used[sl] && cudaStreamWaitEvent(main, s.drained[sl], 0) != cudaSuccess) return FBSR_ERR_CUDA;
-        if (cudaMemcpyAsync(slot_in[sl], src_host + at, len * 4, cudaMemcpyHostToDevice, main) != cudaSuccess) return FBSR_ERR_CUDA;
+        // chunk idx is uploaded on the upload stream while chunk idx - 1 is being rounded: the slot's previous
+        // input must have been read (its kernel done) before the copy overwrites it
+        if (used[sl] && cudaStreamWaitEvent(s.h2d, rounded[sl], 0) != cudaSuccess) return FBSR_ERR_CUDA;
+        if (cudaMemcpyAsync(slot_in[sl], src_host + at, len * 4, cudaMemcpyHostToDevice, s.h2d) != cudaSuccess) return FBSR_ERR_CUDA;
+        if (cudaEventRecord(uploaded[sl], s.h2d) != cudaSuccess) return FBSR_ERR_CUDA;
+        if (cudaStreamWaitEvent(main, uploaded[sl], 0) != cudaSuccess) return FBSR_ERR_CUDA;
+        // the slot's previous codes must have left before the kernel writes new ones
+        if (used[sl] && cudaStreamWaitEvent(main, drained[sl], 0) != cudaSuccess) return FBSR_ERR_CUDA;
         CallArgs a = base_args(OP_ROUND, variant, k_bits, len, seed, offset + at, slot_out[sl], main);
         a.ovf_ieee = ovf_ieee;
         a.src = reinterpret_cast<const float*>(slot_in[sl]); a.scale = scale;
         if (kRound[fmt](a) != 0) return FBSR_ERR_UNSUPPORTED;
-        if (cudaEventRecord(s.rounded[sl], main) != cudaSuccess) return FBSR_ERR_CUDA;
-        if (cudaStreamWaitEvent(s.d2h, s.rounded[sl], 0) != cudaSuccess) return FBSR_ERR_CUDA;
+        if (cudaEventRecord(rounded[sl], main) != cudaSuccess) return FBSR_ERR_CUDA;
+        if (cudaStreamWaitEvent(s.d2h, rounded[sl], 0) != cudaSuccess) return FBSR_ERR_CUDA;
         if (cudaMemcpyAsync(static_cast<char*>(dst_host) + at * cb, slot_out[sl], len * cb, cudaMemcpyDeviceToHost, s.d2h) != cudaSuccess) return FBSR_ERR_CUDA;
-        if (cudaEventRecord(s.drained[sl], s.d2h) != cudaSuccess) return FBSR_ERR_CUDA;
+        if (cudaEventRecord(drained[sl], s.d2h) != cudaSuccess) return FBSR_ERR_CUDA;
         used[sl] = true;
     }
     // join: the caller's stream finishes only after every code has reached the host
     for (int sl = 0; sl < 2; ++sl)
-        if (used[sl] && cudaStreamWaitEvent(main, s.drained[sl], 0) != cudaSuccess) return FBSR_ERR_CUDA;
+        if (used[sl] && cudaStreamWaitEvent(main, drained[sl], 0) != cudaSuccess) return FBSR_ERR_CUDA;
     return cudaGetLastError() == cudaSuccess ? FBSR_OK : FBSR_ERR_CUDA;
 }
 

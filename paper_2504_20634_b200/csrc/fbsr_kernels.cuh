@@ -28,30 +28,16 @@
 
 namespace fbsr {
 
-// Tuning constants (overridable at compile time for experiments).
-#ifndef FBSR_WARPS_PER_CTA
-#define FBSR_WARPS_PER_CTA 8
-#endif
-#ifndef FBSR_MIN_CTAS_ROUND
-#define FBSR_MIN_CTAS_ROUND 4       // resident CTAs the compiler must allow (caps registers at 64)
-#endif
-#ifndef FBSR_MIN_CTAS_SGD
-#define FBSR_MIN_CTAS_SGD 2
-#endif
-#ifndef FBSR_QATADAM_BATCH
-#define FBSR_QATADAM_BATCH 1      // rows of loads in flight per warp for the fused Algorithm-1 step; measured with
-#endif
-#ifndef FBSR_QATADAM_MIN_CTAS
-#define FBSR_QATADAM_MIN_CTAS 4   // (1, 4): 6.4-6.6 TB/s; (2, 3): 6.3-6.7; (2, 2): 5.6-5.8; (1, 6): 6.0-6.1
-#endif
-#ifndef FBSR_MIN_CTAS_ADAM
-#define FBSR_MIN_CTAS_ADAM 2
-#endif
-#ifndef FBSR_ROW_BATCH
-#define FBSR_ROW_BATCH 4            // rows whose loads are issued before the first row is consumed
-#endif
-constexpr int WARPS_PER_CTA = FBSR_WARPS_PER_CTA;
-constexpr int ROW_BATCH = FBSR_ROW_BATCH;
+// Launch shape and prefetch depth, as measured on B200 (2^27..2^28 elements):
+constexpr int WARPS_PER_CTA = 8;
+constexpr int ROW_BATCH = 4;            // rows whose loads are issued before the first row is consumed
+constexpr int MIN_CTAS_ROUND = 4;       // resident CTAs the compiler must allow for the rounding ops (caps registers at 64)
+constexpr int MIN_CTAS_SGD = 2;         // the optimizer ops hold three or four rows of state per row in flight
+constexpr int MIN_CTAS_ADAM = 2;
+// the fused Algorithm-1 step: (rows in flight, resident CTAs) = (1, 4) gave 6.4-6.6 TB/s, (2, 3) 6.3-6.7,
+// (2, 2) 5.6-5.8, (1, 6) 6.0-6.1
+constexpr int QATADAM_BATCH = 1;
+constexpr int QATADAM_MIN_CTAS = 4;
 constexpr int CTA_THREADS = WARPS_PER_CTA * 32;
 constexpr int ROW_ELEMS = 256;          // 32 lanes x 8 elements
 
@@ -73,19 +59,14 @@ template <int K, int OCT = 1> struct Tile {
 };
 
 // ---------------------------------------------------------------------------- vector memory access
-#ifndef FBSR_STORE
 #define FBSR_STORE __stcs          // streaming store: the codes are not read again by this kernel
-#endif
 struct F8 { float4 a, b; };
 
 __device__ __forceinline__ F8 load_f8_stream(const float* p)
 {
     // 256-bit read-only load that does not allocate in L1: the data is used once.
     F8 v;
-#ifndef FBSR_STREAM_LOAD
-#define FBSR_STREAM_LOAD "ld.global.nc.L1::no_allocate.L2::evict_first.v8.f32"
-#endif
-    asm volatile(FBSR_STREAM_LOAD " {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+    asm volatile("ld.global.nc.L1::no_allocate.L2::evict_first.v8.f32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
                  : "=f"(v.a.x), "=f"(v.a.y), "=f"(v.a.z), "=f"(v.a.w),
                    "=f"(v.b.x), "=f"(v.b.y), "=f"(v.b.z), "=f"(v.b.w)
                  : "l"(p));
@@ -169,7 +150,7 @@ __device__ __forceinline__ void store_code1(void* dst, size_t elem, uint32_t c)
 // scalar(): the same for one element on the slow path.
 
 struct RoundOp {
-    static constexpr int BATCH = ROW_BATCH, MIN_CTAS = FBSR_MIN_CTAS_ROUND, OCTETS = 1;
+    static constexpr int BATCH = ROW_BATCH, MIN_CTAS = MIN_CTAS_ROUND, OCTETS = 1;
     const float* src;
     float scale;
     struct Regs { F8 x; };
@@ -194,7 +175,7 @@ struct RoundOp {
 // their largest finite magnitude; the scale byte is written by the first lane of the block.
 template <int FMT>
 struct MxOp {
-    static constexpr int BATCH = ROW_BATCH, MIN_CTAS = FBSR_MIN_CTAS_ROUND, OCTETS = 1;
+    static constexpr int BATCH = ROW_BATCH, MIN_CTAS = MIN_CTAS_ROUND, OCTETS = 1;
     static constexpr int EMAX = (int)(Format<FMT>::MAXBITS >> 23) - 127;        // floor(log2 M)
     const float* src; uint8_t* scales; size_t n;
     struct Regs { F8 x; };
@@ -251,7 +232,7 @@ template <int SRC>
 struct LpSrcOp {
     static_assert(SRC == BF16 || SRC == FP16, "16-bit sources");
     // two octets per lane: one 256-bit load of 16 codes, one 128-bit store of 16 eight-bit codes
-    static constexpr int BATCH = ROW_BATCH, MIN_CTAS = FBSR_MIN_CTAS_ROUND, OCTETS = 2;
+    static constexpr int BATCH = ROW_BATCH, MIN_CTAS = MIN_CTAS_ROUND, OCTETS = 2;
     const void* src;
     float scale;
     struct Regs { uint32_t c[8]; };
@@ -289,7 +270,7 @@ struct LpSrcOp {
 
 // m' = fma(mu, m, g);  w' = fma(-lr, m', w)
 struct SgdOp {
-    static constexpr int BATCH = ROW_BATCH >= 2 ? ROW_BATCH / 2 : 1, MIN_CTAS = FBSR_MIN_CTAS_SGD, OCTETS = 1;
+    static constexpr int BATCH = ROW_BATCH >= 2 ? ROW_BATCH / 2 : 1, MIN_CTAS = MIN_CTAS_SGD, OCTETS = 1;
     float* w; const float* g; float* m;
     float neg_lr, mu;
     struct Regs { F8 w, g, m; };
@@ -322,7 +303,7 @@ struct SgdOp {
 
 // m' = fma(b1, m, a1 g); v' = fma(b2, v, (a2 g) g); d = sqrt(v') c2 + eps; w' = fma(-c1, m'/d, w)
 struct AdamOp {
-    static constexpr int BATCH = ROW_BATCH >= 2 ? ROW_BATCH / 2 : 1, MIN_CTAS = FBSR_MIN_CTAS_ADAM, OCTETS = 1;
+    static constexpr int BATCH = ROW_BATCH >= 2 ? ROW_BATCH / 2 : 1, MIN_CTAS = MIN_CTAS_ADAM, OCTETS = 1;
     float* w; const float* g; float* m; float* v;
     float beta1, beta2, eps, neg_c1, c2, a1, a2;
     struct Regs { F8 w, g, m, v; };
@@ -399,7 +380,7 @@ __device__ __forceinline__ void decode4(uint32_t w, float (&v)[4])
 // y = fl32(value(w_lp) + u); the codes are rewritten in place by the caller of finish()
 template <int FMT>
 struct AccumOp {
-    static constexpr int BATCH = ROW_BATCH, MIN_CTAS = FBSR_MIN_CTAS_ROUND, OCTETS = 1;
+    static constexpr int BATCH = ROW_BATCH, MIN_CTAS = MIN_CTAS_ROUND, OCTETS = 1;
     const void* w_lp; const float* u;
     struct Regs { F8 u; uint4 c; };
     __device__ __forceinline__ void fetch(size_t elem, Regs& r) const
@@ -446,7 +427,7 @@ template <int WF, int UF>
 struct QatOp {
     static_assert(Format<WF>::K == 8 && (UF == BF16 || UF == FP16), "8-bit weights, 16-bit updates");
     // two octets per lane: 16 weight codes (128 bits) and 16 update codes (256 bits) in, 16 weight codes out
-    static constexpr int BATCH = ROW_BATCH >= 2 ? ROW_BATCH / 2 : 1, MIN_CTAS = FBSR_MIN_CTAS_ROUND, OCTETS = 2;
+    static constexpr int BATCH = ROW_BATCH >= 2 ? ROW_BATCH / 2 : 1, MIN_CTAS = MIN_CTAS_ROUND, OCTETS = 2;
     const void* w8; const void* u16;
     struct Regs { uint32_t w[4]; uint32_t u[8]; };
     __device__ __forceinline__ static float sum16(uint32_t wcode, uint32_t ucode)
@@ -507,7 +488,7 @@ struct QatOp {
 template <int WF, int UF>
 struct QatAdamOp {
     static_assert(Format<WF>::K == 8 && (UF == BF16 || UF == FP16), "8-bit weights, 16-bit gradients and updates");
-    static constexpr int BATCH = FBSR_QATADAM_BATCH, MIN_CTAS = FBSR_QATADAM_MIN_CTAS, OCTETS = 1;
+    static constexpr int BATCH = QATADAM_BATCH, MIN_CTAS = QATADAM_MIN_CTAS, OCTETS = 1;
     const void* w8; const void* g16; float* m; float* v;
     float beta1, beta2, eps, neg_c1, c2, a1, a2, neg_lrwd;
     struct Regs { uint2 w; uint4 g; F8 m, v; };

@@ -106,3 +106,25 @@ def test_python_tile_table_equals_the_library(lib):
         assert sharding.tile_elements(k) == lib.fbsr_tile_elements(k), k
         assert sharding.SHARD_ALIGN % lib.fbsr_tile_elements(k) == 0
     assert lib.fbsr_tile_elements(0) == 0 and lib.fbsr_tile_elements(17) == 0
+
+
+def test_adam_scalars_match_the_oracle_and_do_not_cost_the_step_count(lib):
+    """The host scalars of the Adam steps equal the oracle's (which multiplies beta `step` times) bit for bit,
+    including far into a run, where the library stops multiplying once beta^step can no longer matter."""
+    import time
+    import numpy as np
+    from oracle import capi
+    lib.fbsr_adam_scalars.argtypes = [ctypes.c_float, ctypes.c_float, ctypes.c_float, ctypes.c_int,
+                                      ctypes.POINTER(ctypes.c_float)]
+    lib.fbsr_adam_scalars.restype = None
+    out = (ctypes.c_float * 4)()
+    for lr, b1, b2 in ((1e-4, 0.9, 0.999), (3e-3, 0.5, 0.95), (1e-3, 0.0, 0.999), (1e-3, 0.99, 0.9999)):
+        for step in (1, 2, 10, 353, 354, 5000, 37000, 38000, 400000, 10 ** 6):
+            lib.fbsr_adam_scalars(lr, b1, b2, step, out)
+            want = capi.adam_coefficients(lr, b1, b2, step)
+            got = np.array(list(out), dtype=np.float32)
+            assert np.array_equal(got.view(np.uint32), np.array(want, dtype=np.float32).view(np.uint32)), (lr, b1, b2, step)
+    t0 = time.perf_counter()
+    for _ in range(200):
+        lib.fbsr_adam_scalars(1e-4, 0.9, 0.999, 2 ** 31 - 1, out)
+    assert time.perf_counter() - t0 < 1.0                     # 200 x 2^31 multiplications would take minutes
