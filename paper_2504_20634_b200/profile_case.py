@@ -17,7 +17,7 @@ from paper_2504_20634_b200 import workloads
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--op", default="round", choices=["round", "sgd", "adam", "accumulate", "stats", "bits", "lp", "mx", "desc", "qat_adamw"])
+    ap.add_argument("--op", default="round", choices=["round", "sgd", "adam", "accumulate", "stats", "bits", "lp", "mx", "desc", "qat", "qat_adamw"])
     ap.add_argument("--src-fmt", default="bf16", help="source format for --op lp")
     ap.add_argument("--fmt", default="bf16")
     ap.add_argument("--variant", default="srf")
@@ -34,13 +34,13 @@ def main():
     n = 1 << args.log2n
     dev = torch.device("cuda", 0)
     scale = args.scale
+    base_fmt = args.fmt.split("+")[0]               # "fp16+ieee": the IEEE overflow option
     if args.data == "fp8act":
         x, scale = workloads.fp8_activations(base_fmt, rows=n // 32768, cols=32768, device=dev)
     elif args.misalign:
         x = workloads.bandwidth_sweep(n + args.misalign, seed=1234, device=dev)[args.misalign:]
     else:
         x = workloads.bandwidth_sweep(n, seed=1234, device=dev)
-    base_fmt = args.fmt.split("+")[0]               # "fp16+ieee": the IEEE overflow option
     code_bytes = 2 if base_fmt in ("bf16", "fp16") else 1
     out = torch.empty(n, dtype=fbsr.CODE_DTYPE[base_fmt], device=dev)
     if args.op == "round":
@@ -63,6 +63,12 @@ def main():
         bytes_per_elem = 20
         run = lambda s: fbsr.fbsr_qat_adamw_step(out, g16, m, v, args.fmt, args.src_fmt, args.variant, args.k, s, 0,
                                                  1e-3, 0.9, 0.95, 1e-8, 0.1, s + 1)
+    elif args.op == "qat":
+        # last line of Algorithm 1 with the 16-bit sum: 8-bit weights in place, 16-bit updates: 4 B/element
+        fbsr.fbsr_round(x.mul(2.0 ** -18).clamp_(-3, 3), base_fmt, "rtne", 1, seed=0, out=out)
+        u16 = (torch.randn(n, device=dev) * 1e-2).to(torch.bfloat16 if args.src_fmt == "bf16" else torch.float16).view(torch.uint16)
+        bytes_per_elem = 4
+        run = lambda s: fbsr.fbsr_qat_update(out, u16, args.fmt, args.src_fmt, args.variant, args.k, seed=s)
     elif args.op == "lp":
         codes = workloads.lp_sweep(n, args.src_fmt, device=dev)
         bytes_per_elem = 2 + code_bytes
