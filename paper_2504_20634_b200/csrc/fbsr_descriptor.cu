@@ -126,8 +126,10 @@ descriptor_kernel(const float* __restrict__ src, void* __restrict__ dst, const u
 // the generator calls of a tile are shared through the warp's buffer and the fields are taken from the packed
 // word stream, as in the bandwidth kernel; a lane owns 8 consecutive elements of a 256-element row.
 // one_addition: the draw fits under the format's 24 - P excess bits (decided by the host, uniform for the launch).
-template <int VAR, int N, int CODE_BYTES>
-__global__ void __launch_bounds__(CTA_THREADS, 4)
+// ROW_FORM (decided by the host): the draw fits under the excess bits and the code fits above them, so whole
+// lane-rows are rounded by the one-addition form; otherwise every element goes through the element-wise rounder.
+template <int VAR, int N, int CODE_BYTES, bool ROW_FORM>
+__global__ void __launch_bounds__(CTA_THREADS, 3)
 descriptor_tile_kernel(const float* __restrict__ src, const float scale, void* __restrict__ dst, const uint64_t n_tiles,
                        const uint64_t call0, const uint32_t k0, const uint32_t k1, const RtFormat f,
                        const bool ieee_overflow, const bool one_addition)
@@ -148,6 +150,21 @@ descriptor_tile_kernel(const float* __restrict__ src, const float scale, void* _
     const uint32_t max_pattern = f.MAXCODE << sh0;
     const uint32_t fast_limit = ieee_overflow ? f.MAXBITS : 0x7F7FFFFFu;
     const uint32_t sign_shift = 32u - (uint32_t)(8 * CODE_BYTES);
+    // Row form, as in the bandwidth kernel: the saturated pattern is moved left so that the code comes out of the
+    // addition in the top K bits (packing is then byte selection), the draw is rotated to where it is added and
+    // masked there, and Inf / NaN are found per lane-row by a floating-point flag and redone element by element.
+    // It needs the code to fit above the excess bits (32 - K - sh0 >= 0: every format with at most 8 exponent bits).
+    constexpr int KBITS = 8 * CODE_BYTES;
+    const int lift = 32 - KBITS - sh0;                        // left shift of the pattern
+    constexpr bool row_form = ROW_FORM;
+    const uint32_t lift_mul = row_form ? 1u << lift : 1u;
+    const int draw_pos = pos + (row_form ? lift : 0);         // bit where the draw's lowest bit is added
+    const uint32_t draw_mask = DRAWS ? ((1u << N) - 1u) << draw_pos : 0u;
+    const uint32_t half_l = half * lift_mul, below_half_l = below_half * lift_mul;
+    const float tie = __uint_as_float(f.MAXBITS + (1u << (sh0 - 1)));          // M + ulp(M) / 2
+    const bool tie_overflows = (f.MAXCODE & 1u) != 0u;
+    const uint32_t overflow_top = (f.HAS_INF ? f.INFCODE : f.NANCODE) << (32 - KBITS);
+    const uint32_t zero_mask = f.SINGLE_ZERO ? 0xFFFFFFFFu : 0u;
 
     for (uint64_t tile = (uint64_t)blockIdx.x * WARPS_PER_CTA + warp; tile < n_tiles;
          tile += (uint64_t)gridDim.x * WARPS_PER_CTA) {
@@ -186,13 +203,69 @@ descriptor_tile_kernel(const float* __restrict__ src, const float scale, void* _
                 } else {
                     d.from_normalised(wb, p0);
                 }
+                if constexpr (row_form) {
+                    float y[8], flag = 0.0f;
+                    uint32_t t[8];
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) {
+                        y[c] = __fmul_rn(x[c], scale);
+                        flag = __fmaf_rn(y[c], 0.0f, flag);                      // NaN iff y is Inf or NaN
+                        uint32_t u = __float_as_uint(__fmul_rz(fabsf(y[c]), rescale));
+                        if constexpr (STICKY) u |= (u ^ __float_as_uint(__fmul_ru(fabsf(y[c]), rescale))) & 1u;
+                        u = min(u, max_pattern);
+                        const uint32_t base = u * lift_mul;
+                        uint32_t draw = 0u;
+                        if constexpr (DRAWS) {
+                            // the field of element c sits at bit b of its word: rotate it to draw_pos and mask it there
+                            constexpr int G = Draws8<N>::G;
+                            const int b = (c % G) * N;
+                            draw = __funnelshift_l(d.u[c / G], d.u[c / G], (uint32_t)(draw_pos - b) & 31u) & draw_mask;
+                        }
+                        if constexpr (VAR == SRFF) t[c] = base + draw;
+                        else if constexpr (VAR == SRF) t[c] = base + half_l + draw;
+                        else if constexpr (VAR == RTA) t[c] = base + half_l;
+                        else t[c] = base + below_half_l + ((((u >> pos) & 1u) ^ (VAR == RTO ? 1u : 0u)) * lift_mul) + draw;
+                        if (ieee_overflow) {
+                            const bool beyond = tie_overflows ? fabsf(y[c]) >= tie : fabsf(y[c]) > tie;
+                            t[c] = beyond ? overflow_top : t[c];
+                        }
+                    }
+                    if (flag == flag) {
+                        // codes in the top K bits, bit 31 clear: pack by byte selection, signs from y
+                        if constexpr (CODE_BYTES == 2) {
+                            uint32_t w[4];
+#pragma unroll
+                            for (int q = 0; q < 4; ++q) {
+                                const uint32_t cw = __byte_perm(t[2 * q], t[2 * q + 1], 0x7632);
+                                uint32_t sg = __byte_perm(__float_as_uint(y[2 * q]), __float_as_uint(y[2 * q + 1]), 0x7632) & 0x80008000u;
+                                sg &= ~zero_mask | (cw + 0x7FFF7FFFu);                // one zero only: a zero magnitude takes no sign
+                                w[q] = cw | sg;
+                            }
+                            store_words<4>(static_cast<char*>(dst) + (e0 + p0) * 2, w);
+                        } else {
+                            uint32_t w[2];
+#pragma unroll
+                            for (int q = 0; q < 2; ++q) {
+                                const uint32_t c01 = __byte_perm(t[4 * q], t[4 * q + 1], 0x7373), c23 = __byte_perm(t[4 * q + 2], t[4 * q + 3], 0x7373);
+                                const uint32_t s01 = __byte_perm(__float_as_uint(y[4 * q]), __float_as_uint(y[4 * q + 1]), 0x7373);
+                                const uint32_t s23 = __byte_perm(__float_as_uint(y[4 * q + 2]), __float_as_uint(y[4 * q + 3]), 0x7373);
+                                const uint32_t cw = __byte_perm(c01, c23, 0x5410);
+                                uint32_t sg = __byte_perm(s01, s23, 0x5410) & 0x80808080u;
+                                sg &= ~zero_mask | (cw + 0x7F7F7F7Fu);
+                                w[q] = cw | sg;
+                            }
+                            store_words<2>(static_cast<char*>(dst) + (e0 + p0), w);
+                        }
+                        continue;
+                    }
+                }
                 uint32_t codes[8];
 #pragma unroll
                 for (int c = 0; c < 8; ++c) {
                     const uint32_t yb = __float_as_uint(__fmul_rn(x[c], scale));    // a NaN takes the other branch
                     const uint32_t mbits = yb & 0x7FFFFFFFu;
                     const uint32_t nr = DRAWS ? d.template at<0>(c) : 0u;
-                    if (one_addition && mbits <= fast_limit) {
+                    if (!row_form && one_addition && mbits <= fast_limit) {
                         const float mag = __uint_as_float(mbits);
                         uint32_t u = __float_as_uint(__fmul_rz(mag, rescale));
                         if constexpr (STICKY) u |= (u ^ __float_as_uint(__fmul_ru(mag, rescale))) & 1u;
@@ -235,13 +308,11 @@ void launch_descriptor_tiles(const TileCall& t)
 {
     const uint64_t want = (t.n_tiles + WARPS_PER_CTA - 1) / WARPS_PER_CTA;
     const unsigned grid = (unsigned)(want < 0x7FFFFFF0ull ? want : 0x7FFFFFF0ull);
-    if (t.f.K == 16) {
-        descriptor_tile_kernel<VAR, N, 2><<<grid, CTA_THREADS, 0, t.stream>>>(t.src, t.scale, t.dst, t.n_tiles, t.call0, t.k0,
-                                                                            t.k1, t.f, t.ieee_overflow, t.one_addition);
-    } else {
-        descriptor_tile_kernel<VAR, N, 1><<<grid, CTA_THREADS, 0, t.stream>>>(t.src, t.scale, t.dst, t.n_tiles, t.call0, t.k0,
-                                                                            t.k1, t.f, t.ieee_overflow, t.one_addition);
-    }
+    const bool row_form = t.one_addition && 32 - t.f.K - (24 - t.f.P) >= 0;
+    auto kern = t.f.K == 16 ? (row_form ? descriptor_tile_kernel<VAR, N, 2, true> : descriptor_tile_kernel<VAR, N, 2, false>)
+                            : (row_form ? descriptor_tile_kernel<VAR, N, 1, true> : descriptor_tile_kernel<VAR, N, 1, false>);
+    kern<<<grid, CTA_THREADS, 0, t.stream>>>(t.src, t.scale, t.dst, t.n_tiles, t.call0, t.k0, t.k1, t.f, t.ieee_overflow,
+                                             t.one_addition);
     count_launch();
 }
 
