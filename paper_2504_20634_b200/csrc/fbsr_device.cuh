@@ -338,7 +338,13 @@ template <int FMT, int VAR, int N> struct FastRow {
                     : (VAR == SRFF ? N <= SH0 : VAR == SRF ? N <= SH0 - 1 : N <= SH0 - 2);
 };
 
-template <int FMT, int VAR, int N>
+// VALUE_BITS: an upper bound on the significant bits of the values handed in (24 for arbitrary binary32 values; 8 or
+// 11 when they are exactly bfloat16 or binary16 values).  A value of b bits loses bits in the rescaled pattern only
+// when it lies b + 8 or more binades below the target's emin, where the pattern is below 2^(b - 1); the nearest-even
+// pre-round of SRC (and the deterministic modes) looks at the lost bits only to tell a tie at bit POS - 1 from a value
+// just above it, and a pattern below 2^(b - 1) is below every such tie once POS >= b: the sticky bit (a second,
+// upward-rounded multiply per element) is then never needed.
+template <int FMT, int VAR, int N, int VALUE_BITS = 24>
 __device__ __forceinline__ bool round_row_fast(const float (&y)[8], const Draws8<N>& d, uint32_t (&t)[8])
 {
     using F = Format<FMT>;
@@ -417,7 +423,7 @@ __device__ __forceinline__ bool round_row_fast(const float (&y)[8], const Draws8
         } else {
             const float rescale = __uint_as_float((uint32_t)(128 - F::EMINB) << 23);   // 2^(1 - EMINB)
             u = __float_as_uint(__fmul_rz(fabsf(y[c]), rescale));
-            if constexpr (EFF == SRC || EFF == RTNE || EFF == RTO) {
+            if constexpr ((EFF == SRC || EFF == RTNE || EFF == RTO) && POS < VALUE_BITS) {
                 const uint32_t up = __float_as_uint(__fmul_ru(fabsf(y[c]), rescale));
                 u |= (u ^ up) & 1u;                           // sticky: round to odd
             }

@@ -3,6 +3,7 @@
 // scales, 5 = rounding with statistics (three units so that they compile in parallel), 1 = fused optimizer and
 // accumulation, 2 = 16-bit sources and the 16-bit-sum update, 3 = the fused Algorithm-1 step (2, 3: 8-bit targets only).
 #include <array>
+#include <cmath>
 #include <utility>
 
 #include "fbsr_internal.h"
@@ -59,11 +60,11 @@ template <int UF> inline QatAdamOp<QAT_WF, UF> op_advance(QatAdamOp<QAT_WF, UF> 
 {
     o.w8 = static_cast<const uint8_t*>(o.w8) + h; o.g16 = static_cast<const uint16_t*>(o.g16) + h; o.m += h; o.v += h; return o;
 }
-template <int SRC> inline bool op_aligned(const LpSrcOp<SRC>& o, size_t h)
+template <int SRC, bool P2> inline bool op_aligned(const LpSrcOp<SRC, P2>& o, size_t h)
 {
     return aligned(static_cast<const uint16_t*>(o.src) + h, 32);
 }
-template <int SRC> inline LpSrcOp<SRC> op_advance(LpSrcOp<SRC> o, size_t h)
+template <int SRC, bool P2> inline LpSrcOp<SRC, P2> op_advance(LpSrcOp<SRC, P2> o, size_t h)
 {
     o.src = static_cast<const uint16_t*>(o.src) + h; return o;
 }
@@ -148,7 +149,7 @@ Plan make_plan(const Op& op, const CallArgs& a)
 // listed here (plain rounding with generated draws, 16-bit sources); the other calls use the general kernel.
 template <class Op, bool BITS> struct HasIeee { static constexpr bool value = false; };
 template <> struct HasIeee<RoundOp, false> { static constexpr bool value = true; };
-template <int SRC> struct HasIeee<LpSrcOp<SRC>, false> { static constexpr bool value = true; };
+template <int SRC, bool P2> struct HasIeee<LpSrcOp<SRC, P2>, false> { static constexpr bool value = true; };
 
 template <class Op, int VAR, int K, bool BITS>
 int run(const Op& op, const CallArgs& a)
@@ -290,8 +291,18 @@ int FBSR_CAT(dispatch_lp_, FBSR_FMT)(const CallArgs& a)
         if (a.src_fmt == FP16) return by_variant_and_k<QatOp<FMT, FP16>, false>(QatOp<FMT, FP16>{a.dst, a.src_lp}, a);
         return 1;
     }
-    if (a.src_fmt == BF16) return by_variant_and_k<LpSrcOp<BF16>, false>(LpSrcOp<BF16>{a.src_lp, a.scale}, a);
-    if (a.src_fmt == FP16) return by_variant_and_k<LpSrcOp<FP16>, false>(LpSrcOp<FP16>{a.src_lp, a.scale}, a);
+    // a power-of-two scale keeps the source's 8 or 11 significant bits: the kernels that round to nearest first
+    // (SRC and the deterministic modes) then need no sticky bit; the other variants have no such code to drop
+    int exponent = 0;
+    const bool pow2 = std::frexp(a.scale, &exponent) == 0.5f && (a.variant == SRC || a.variant >= RTNE);
+    if (a.src_fmt == BF16) {
+        if (pow2) return by_variant_and_k<LpSrcOp<BF16, true>, false>(LpSrcOp<BF16, true>{a.src_lp, a.scale}, a);
+        return by_variant_and_k<LpSrcOp<BF16>, false>(LpSrcOp<BF16>{a.src_lp, a.scale}, a);
+    }
+    if (a.src_fmt == FP16) {
+        if (pow2) return by_variant_and_k<LpSrcOp<FP16, true>, false>(LpSrcOp<FP16, true>{a.src_lp, a.scale}, a);
+        return by_variant_and_k<LpSrcOp<FP16>, false>(LpSrcOp<FP16>{a.src_lp, a.scale}, a);
+    }
     return 1;
 }
 #elif FBSR_GROUP == 3

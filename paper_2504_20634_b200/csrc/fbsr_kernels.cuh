@@ -227,10 +227,16 @@ struct MxOp {
     }
 };
 
-// Source already in a 16-bit format: widen exactly (Eq. (1)), then scale.
-template <int SRC>
+// Significant bits of the values an op hands to the row rounder: 24 unless the op declares VALUE_BITS.
+template <class Op, class = void> struct ValueBits { static constexpr int value = 24; };
+template <class Op> struct ValueBits<Op, decltype((void)Op::VALUE_BITS)> { static constexpr int value = Op::VALUE_BITS; };
+
+// Source already in a 16-bit format: widen exactly (Eq. (1)), then scale.  POW2_SCALE (decided by the host): the
+// scale is a power of two, so the scaled value still has the source's 8 or 11 significant bits.
+template <int SRC, bool POW2_SCALE = false>
 struct LpSrcOp {
     static_assert(SRC == BF16 || SRC == FP16, "16-bit sources");
+    static constexpr int VALUE_BITS = POW2_SCALE ? (SRC == BF16 ? 8 : 11) : 24;
     // two octets per lane: one 256-bit load of 16 codes, one 128-bit store of 16 eight-bit codes
     static constexpr int BATCH = ROW_BATCH, MIN_CTAS = MIN_CTAS_ROUND, OCTETS = 2;
     const void* src;
@@ -426,6 +432,7 @@ struct AccumOp {
 template <int WF, int UF>
 struct QatOp {
     static_assert(Format<WF>::K == 8 && (UF == BF16 || UF == FP16), "8-bit weights, 16-bit updates");
+    static constexpr int VALUE_BITS = UF == BF16 ? 8 : 11;              // the sum is a value of the 16-bit format
     // two octets per lane: 16 weight codes (128 bits) and 16 update codes (256 bits) in, 16 weight codes out
     static constexpr int BATCH = ROW_BATCH >= 2 ? ROW_BATCH / 2 : 1, MIN_CTAS = MIN_CTAS_ROUND, OCTETS = 2;
     const void* w8; const void* u16;
@@ -488,6 +495,7 @@ struct QatOp {
 template <int WF, int UF>
 struct QatAdamOp {
     static_assert(Format<WF>::K == 8 && (UF == BF16 || UF == FP16), "8-bit weights, 16-bit gradients and updates");
+    static constexpr int VALUE_BITS = UF == BF16 ? 8 : 11;              // the sum is a value of the 16-bit format
     static constexpr int BATCH = QATADAM_BATCH, MIN_CTAS = QATADAM_MIN_CTAS, OCTETS = 1;
     const void* w8; const void* g16; float* m; float* v;
     float beta1, beta2, eps, neg_c1, c2, a1, a2, neg_lrwd;
@@ -715,7 +723,7 @@ tile_kernel(const Op op, void* __restrict__ dst, const uint64_t n_tiles, const u
                             d.from_normalised(wb, po);
                         }
                         uint32_t t[8];
-                        const bool redo = round_row_fast<FMT, VAR, K>(y, d, t);
+                        const bool redo = round_row_fast<FMT, VAR, K, ValueBits<Op>::value>(y, d, t);
                         if constexpr (IEEE && FMT != BF16) {
 #pragma unroll
                             for (int i = 0; i < 8; ++i)

@@ -83,3 +83,18 @@ def test_large_lp_sweep_sampled():
             for (a, b), h in zip(slices, hs):
                 gu.assert_codes_equal(out[a:b], capi.fbsr_round_lp(h, "bf16", dst_fmt, variant, k, seed=5, offset=a),
                                       "%s %s k=%d at %d" % (dst_fmt, variant, k, a))
+
+
+@pytest.mark.parametrize("src_fmt", ["bf16", "fp16"])
+def test_power_of_two_scales_with_nearest_first_variants(src_fmt):
+    """With a power-of-two scale the kernels that round to nearest first (SRC, ties to even / odd) drop the sticky
+    bit, because a 16-bit value loses bits in the rescaled pattern only far below every tie: every source code, scales
+    that push the values deep below and far above the targets' ranges (and into binary32's own subnormals)."""
+    codes = np.arange(1 << 16, dtype=np.uint16)
+    cd = gu.from_np_codes(codes)
+    for dst_fmt in ("e4m3", "e5m2", "b8p4"):
+        for scale in (2.0 ** -30, 2.0 ** -13, 2.0 ** -7, 0.5, 2.0 ** 9, 2.0 ** 40, 2.0 ** -120):
+            for variant, k in (("src", 1), ("src", 3), ("src", 8), ("src", 12), ("src", 13), ("src", 16), ("rtne", 1), ("rto", 1)):
+                got = fbsr.fbsr_round_lp(cd, src_fmt, dst_fmt, variant, k, seed=77, offset=0, scale=scale)
+                expect = capi.fbsr_round_lp(codes, src_fmt, dst_fmt, variant, k, seed=77, offset=0, scale=scale)
+                gu.assert_codes_equal(got, expect, "%s->%s %s k=%d scale=%g" % (src_fmt, dst_fmt, variant, k, scale))
