@@ -23,10 +23,10 @@ HEADERS = ["fbsr_device.cuh", "fbsr_kernels.cuh", "fbsr_internal.h", os.path.joi
 
 def _units():
     units = [("fbsr_api.o", "fbsr_api.cu", []), ("fbsr_descriptor.o", "fbsr_descriptor.cu", [])]
-    for fmt in range(5):
-        for group in (5, 0, 4, 1, 2, 3):      # the longest compilations first
-            if group in (2, 3) and fmt < 2:
-                continue                      # 16-bit sources and the Algorithm-1 step go to the 8-bit targets only
+    for group in (2, 6, 5, 3, 1, 0, 4):       # the longest compilations first
+        for fmt in range(5):
+            if group in (2, 3, 6) and fmt < 2:
+                continue                      # 16-bit sources and the Algorithm-1 steps go to the 8-bit targets only
             units.append(("fbsr_dispatch_f%d_g%d.o" % (fmt, group), "fbsr_dispatch.cu",
                           ["-DFBSR_FMT=%d" % fmt, "-DFBSR_GROUP=%d" % group]))
     return units

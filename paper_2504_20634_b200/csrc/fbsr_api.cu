@@ -22,6 +22,7 @@ const dispatch_fn kOptim[5] = {dispatch_optim_0, dispatch_optim_1, dispatch_opti
 inline bool eight_bit(int fmt) { return fmt == FBSR_E4M3 || fmt == FBSR_E5M2 || fmt == FBSR_B8P4; }
 inline int dispatch_lp(int fmt, const CallArgs& a)
 {
+    if (a.op == OP_QAT) return fmt == FBSR_E4M3 ? dispatch_qat_2(a) : fmt == FBSR_E5M2 ? dispatch_qat_3(a) : dispatch_qat_4(a);
     return fmt == FBSR_E4M3 ? dispatch_lp_2(a) : fmt == FBSR_E5M2 ? dispatch_lp_3(a) : dispatch_lp_4(a);
 }
 

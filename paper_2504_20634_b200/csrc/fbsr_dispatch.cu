@@ -1,7 +1,7 @@
 // Kernel instantiations and launch logic for one target format and one group of
 // operations.  Compiled once per (FBSR_FMT, FBSR_GROUP): FBSR_GROUP 0 = fbsr_round, 4 = supplied bits and block
 // scales, 5 = rounding with statistics (three units so that they compile in parallel), 1 = fused optimizer and
-// accumulation, 2 = 16-bit sources and the 16-bit-sum update, 3 = the fused Algorithm-1 step (2, 3: 8-bit targets only).
+// accumulation, 2 = 16-bit sources, 6 = the 16-bit-sum update, 3 = the fused Algorithm-1 step (2, 3, 6: 8-bit targets only).
 #include <array>
 #include <cmath>
 #include <utility>
@@ -13,7 +13,7 @@
 #error "compile with -DFBSR_FMT=0..4"
 #endif
 #ifndef FBSR_GROUP
-#error "compile with -DFBSR_GROUP=0..5"
+#error "compile with -DFBSR_GROUP=0..6"
 #endif
 
 namespace fbsr {
@@ -286,11 +286,6 @@ int FBSR_CAT(dispatch_round_words_, FBSR_FMT)(const CallArgs& a)
 int FBSR_CAT(dispatch_lp_, FBSR_FMT)(const CallArgs& a)
 {
     static_assert(CODE_BYTES == 1, "16-bit sources are rounded to 8-bit targets");
-    if (a.op == OP_QAT) {
-        if (a.src_fmt == BF16) return by_variant_and_k<QatOp<FMT, BF16>, false>(QatOp<FMT, BF16>{a.dst, a.src_lp}, a);
-        if (a.src_fmt == FP16) return by_variant_and_k<QatOp<FMT, FP16>, false>(QatOp<FMT, FP16>{a.dst, a.src_lp}, a);
-        return 1;
-    }
     // a power-of-two scale keeps the source's 8 or 11 significant bits: the kernels that round to nearest first
     // (SRC and the deterministic modes) then need no sticky bit; the other variants have no such code to drop
     int exponent = 0;
@@ -303,6 +298,14 @@ int FBSR_CAT(dispatch_lp_, FBSR_FMT)(const CallArgs& a)
         if (pow2) return by_variant_and_k<LpSrcOp<FP16, true>, false>(LpSrcOp<FP16, true>{a.src_lp, a.scale}, a);
         return by_variant_and_k<LpSrcOp<FP16>, false>(LpSrcOp<FP16>{a.src_lp, a.scale}, a);
     }
+    return 1;
+}
+#elif FBSR_GROUP == 6
+int FBSR_CAT(dispatch_qat_, FBSR_FMT)(const CallArgs& a)
+{
+    static_assert(CODE_BYTES == 1, "the weights of Algorithm 1 are 8 bits wide");
+    if (a.src_fmt == BF16) return by_variant_and_k<QatOp<FMT, BF16>, false>(QatOp<FMT, BF16>{a.dst, a.src_lp}, a);
+    if (a.src_fmt == FP16) return by_variant_and_k<QatOp<FMT, FP16>, false>(QatOp<FMT, FP16>{a.dst, a.src_lp}, a);
     return 1;
 }
 #elif FBSR_GROUP == 3

@@ -47,6 +47,7 @@ constexpr int MAX_SLOW_GRID = 148 * 8;      // CTAs of the general kernel; also 
     int dispatch_stats_##fmt(const CallArgs&); \
     int dispatch_optim_##fmt(const CallArgs&);\
     int dispatch_lp_##fmt(const CallArgs&); \
+    int dispatch_qat_##fmt(const CallArgs&); \
     int dispatch_qat_adamw_##fmt(const CallArgs&);
 FBSR_DECLARE_DISPATCH(0) FBSR_DECLARE_DISPATCH(1) FBSR_DECLARE_DISPATCH(2) FBSR_DECLARE_DISPATCH(3) FBSR_DECLARE_DISPATCH(4)
 #undef FBSR_DECLARE_DISPATCH
