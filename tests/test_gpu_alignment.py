@@ -65,3 +65,23 @@ def test_ieee_overflow_on_whole_tiles_for_every_draw_width(fmt):
             got = fbsr.fbsr_round(xd, fmt + "+ieee", variant, k, seed=9, offset=2 * tile)
             gu.assert_codes_equal(got, capi.fbsr_round(x, fmt + "+ieee", variant, k, seed=9, offset=2 * tile),
                                   "%s ieee %s k=%d" % (fmt, variant, k))
+
+
+def test_an_lp_call_aligned_as_documented_takes_the_tiled_path():
+    """fbsr_round_lp: source 32-byte aligned, codes 16-byte aligned, offset on the tile grid -> one launch of the tiled
+    kernel for the whole call; a source that is only 16-byte aligned falls to the general kernel, still one launch, and
+    gives the same codes."""
+    tile = 2 * fbsr.fbsr_tile_elements(3)                 # 16 codes per lane: the tiles of this entry point are twice as long
+    n = 6 * tile + 5
+    codes = torch.randint(0, 1 << 15, (n + 16,), device="cuda", dtype=torch.int32).to(torch.uint16)
+    assert codes.data_ptr() % 32 == 0
+    out = torch.empty(n, dtype=torch.uint8, device="cuda")
+    before = fbsr.fbsr_launch_count()
+    fbsr.fbsr_round_lp(codes[:n], "bf16", "e4m3", "src", 3, seed=4, offset=3 * tile, out=out)
+    assert fbsr.fbsr_launch_count() - before == 1
+    expect = capi.fbsr_round_lp(gu.to_np(codes[:n]), "bf16", "e4m3", "src", 3, seed=4, offset=3 * tile)
+    gu.assert_codes_equal(out, expect, "aligned lp call")
+    out2 = torch.empty(n, dtype=torch.uint8, device="cuda")
+    fbsr.fbsr_round_lp(codes[8:8 + n], "bf16", "e4m3", "src", 3, seed=4, offset=3 * tile, out=out2)      # 16 bytes off
+    gu.assert_codes_equal(out2, capi.fbsr_round_lp(gu.to_np(codes[8:8 + n]), "bf16", "e4m3", "src", 3, seed=4, offset=3 * tile),
+                          "lp call 16 bytes off")
