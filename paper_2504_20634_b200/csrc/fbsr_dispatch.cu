@@ -117,6 +117,18 @@ int launch_generic(const Op& op, const CallArgs& a, size_t i_begin, size_t i_end
     uint64_t ctas = (n_calls + CTA_THREADS - 1) / CTA_THREADS;
     if (ctas > (uint64_t)MAX_SLOW_GRID) ctas = MAX_SLOW_GRID;
     const uint64_t dpw = 32u / (unsigned)a.k;
+    if constexpr (!STATS) {
+        // a warp per 32 calls, coalesced accesses
+        uint64_t warps = (n_calls + 31) / 32;
+        ctas = (warps + WARPS_PER_CTA - 1) / WARPS_PER_CTA;
+        if (ctas > (uint64_t)MAX_SLOW_GRID) ctas = MAX_SLOW_GRID;
+        general_coalesced_kernel<Op, FMT, BITS><<<(unsigned)ctas, CTA_THREADS, 0, a.stream>>>(
+            op, a.dst, i_begin, i_end, off, a.variant, a.k, (uint32_t)a.seed, (uint32_t)(a.seed >> 32), a.words,
+            BITS ? (a.n + dpw - 1) / dpw : 0, (uint32_t)(0x100000000ull / dpw) + 1u, a.ovf_ieee);
+        count_launch();
+        if (n_ctas_out) *n_ctas_out = (int)ctas;
+        return 0;
+    }
     generic_kernel<Op, FMT, BITS, STATS><<<(unsigned)ctas, CTA_THREADS, 0, a.stream>>>(
         op, a.dst, i_begin, i_end, off, a.variant, a.k, (uint32_t)a.seed, (uint32_t)(a.seed >> 32),
         a.words, BITS ? (a.n + dpw - 1) / dpw : 0, STATS ? a.group_size : 0, a.gsum_e, a.gsum_e2,

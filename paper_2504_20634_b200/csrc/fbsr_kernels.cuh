@@ -1,6 +1,6 @@
 // Kernels for few-bit stochastic rounding on sm_100a.
 //
-// Two kernels serve every entry point:
+// Kernels:
 //
 //  * tile_kernel: the bandwidth path.  A warp owns a tile of ROWS rows of 256
 //    consecutive elements; in each row a lane owns 8 consecutive elements, so a
@@ -13,9 +13,15 @@
 //    fields of its own elements.  With two draws per word a Philox call serves
 //    exactly one lane's 8 elements and the buffer is skipped.
 //
-//  * generic_kernel: any pointer alignment, any offset, heads and tails.  One
-//    thread per Philox call, scalar loads and stores, run-time k and variant,
-//    optional statistics.
+//  * general_coalesced_kernel / generic_kernel: any pointer alignment, any offset, heads and
+//    tails, scalar loads and stores, run-time k and variant.  The first (no statistics) gives a
+//    warp 32 generator calls and walks their elements 32 at a time, so accesses are coalesced;
+//    the second (with statistics, used for the edges of the statistics call) gives each thread
+//    one call.
+//
+//  * staged_tile_kernel (fbsr_round with pointers of any element alignment), stats_tile_kernel
+//    (rounding plus integer error sums): the tile structure of tile_kernel, described where
+//    they are defined.
 //
 // An "Op" supplies the value to be rounded: the scaled input (fbsr_round), the
 // freshly updated master weight (SGD-momentum, Adam) or the widened stored
@@ -1017,6 +1023,58 @@ generic_kernel(const Op op, void* __restrict__ dst, const uint64_t i_begin, cons
     if constexpr (STATS) {
         stats_cta_reduce(acc);
         if (threadIdx.x == 0) partials[blockIdx.x] = acc;
+    }
+}
+
+// The general kernel without statistics, with coalesced accesses.  A warp takes 32 consecutive generator calls
+// (32 E elements): lane l computes call l of the chunk into the warp's shared buffer, then the warp walks the chunk's
+// elements 32 at a time, lane l taking element 32 j + l, so that a warp instruction reads and writes consecutive
+// elements whatever the pointers' alignment (one thread per call, as in generic_kernel, puts E elements between
+// neighbouring lanes).  Run-time k and variant; elements outside [i_begin, i_end) are skipped.
+// dpw_magic = floor(2^32 / dpw) + 1: the high half of p * dpw_magic is p / dpw for every p below 4096.
+template <class Op, int FMT, bool BITS>
+__global__ void __launch_bounds__(CTA_THREADS)
+general_coalesced_kernel(const Op op, void* __restrict__ dst, const uint64_t i_begin, const uint64_t i_end,
+                         const uint64_t offset, const int variant, const int k, const uint32_t k0, const uint32_t k1,
+                         const uint32_t* __restrict__ words, const uint64_t n_words, const uint32_t dpw_magic,
+                         const int ieee_overflow)
+{
+    const uint32_t dpw = 32u / (uint32_t)k, E = 4u * dpw, mask = (1u << k) - 1u;
+    const bool draws = variant < RTNE;
+    const uint64_t g_first = offset + i_begin, g_last = offset + i_end;     // [g_first, g_last)
+    const uint64_t call_first = g_first / E;
+    const uint64_t n_calls = g_first < g_last ? (g_last - 1) / E - call_first + 1 : 0;
+    const uint64_t n_chunks = (n_calls + 31) / 32;
+    __shared__ __align__(16) uint32_t callbuf[WARPS_PER_CTA][128];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    uint32_t* wb = callbuf[warp];
+    for (uint64_t chunk = (uint64_t)blockIdx.x * WARPS_PER_CTA + warp; chunk < n_chunks;
+         chunk += (uint64_t)gridDim.x * WARPS_PER_CTA) {
+        const uint64_t call = call_first + chunk * 32 + lane;
+        uint4 o = make_uint4(0u, 0u, 0u, 0u);
+        if (draws && call < call_first + n_calls) {
+            if constexpr (BITS) {
+                o.x = call * 4 + 0 < n_words ? words[call * 4 + 0] : 0u;
+                o.y = call * 4 + 1 < n_words ? words[call * 4 + 1] : 0u;
+                o.z = call * 4 + 2 < n_words ? words[call * 4 + 2] : 0u;
+                o.w = call * 4 + 3 < n_words ? words[call * 4 + 3] : 0u;
+            } else {
+                o = philox_block(call, k0, k1);
+            }
+        }
+        *reinterpret_cast<uint4*>(wb + 4 * lane) = o;
+        __syncwarp();
+        const uint64_t g0 = (call_first + chunk * 32) * E;                  // global index of the chunk's first element
+        for (uint32_t p = lane; p < 32u * E; p += 32u) {
+            const uint64_t g = g0 + p;
+            if (g >= g_first && g < g_last) {
+                const uint32_t w = __umulhi(p, dpw_magic), f = p - w * dpw;
+                const uint32_t n = (wb[w] >> (f * (uint32_t)k)) & mask;
+                const uint64_t i = g - offset;
+                store_code1<FMT>(dst, i, round_core<FMT, false>(op.scalar(i), n, variant, k, nullptr, ieee_overflow != 0));
+            }
+        }
+        __syncwarp();                                        // the buffer is rewritten by the next chunk
     }
 }
 
