@@ -131,7 +131,7 @@ def test_ieee_overflow_option(fmt):
 
 
 def test_ieee_overflow_option_with_supplied_bits_and_16_bit_sources():
-    """The same option through fbsr_round_bits and fbsr_round_lp (tiled pass, then the pass that rewrites values beyond M)."""
+    """The same option through fbsr_round_bits and fbsr_round_lp (the tiled IEEE variant for 16-bit sources, the general kernel for supplied bits)."""
     rng = np.random.default_rng(99)
     n = 9 * 1280 + 301
     x = (np.float32(448.0) * (1.0 + rng.uniform(-0.3, 0.3, n))).astype(np.float32) * np.where(rng.integers(0, 2, n), 1, -1).astype(np.float32)
