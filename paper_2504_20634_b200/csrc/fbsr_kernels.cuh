@@ -205,11 +205,22 @@ struct MxOp {
     {
         float x[8];
         unpack(r.x, x);
+        // largest magnitude pattern of the block, Inf and NaN included at first: they are rare, and a block that holds
+        // one (its four lanes see the same maximum, so they decide alike) repeats the reduction over finite values only
         uint32_t m = 0u;
 #pragma unroll
-        for (int c = 0; c < 8; ++c) m = max(m, finite_magnitude(x[c]));
+        for (int c = 0; c < 8; ++c) m = max(m, __float_as_uint(x[c]) & 0x7FFFFFFFu);
         m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, 1));
         m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, 2));
+        const bool special = m >= 0x7F800000u;
+        const uint32_t redo_lanes = __ballot_sync(0xFFFFFFFFu, special);
+        if (special) {
+            m = 0u;
+#pragma unroll
+            for (int c = 0; c < 8; ++c) m = max(m, finite_magnitude(x[c]));
+            m = max(m, __shfl_xor_sync(redo_lanes, m, 1));
+            m = max(m, __shfl_xor_sync(redo_lanes, m, 2));
+        }
         const int e_blk = block_exponent(m);
         const float s = inverse_scale(e_blk);
 #pragma unroll
@@ -362,9 +373,11 @@ __device__ __forceinline__ void decode4(uint32_t w, float (&v)[4])
     if constexpr (FMT == B8P4) {
         asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h01) : "h"((unsigned short)(w & 0xFFFFu)));
         asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h23) : "h"((unsigned short)(w >> 16)));
-        const float2 a = __half22float2(*reinterpret_cast<const __half2*>(&h01));
-        const float2 b = __half22float2(*reinterpret_cast<const __half2*>(&h23));
-        v[0] = __fmul_rn(a.x, 0.5f); v[1] = __fmul_rn(a.y, 0.5f); v[2] = __fmul_rn(b.x, 0.5f); v[3] = __fmul_rn(b.y, 0.5f);
+        // the halving is exact in binary16 as well (the smallest E4M3 value is 2^-9), and there it takes two at a time
+        const __half2 half = __float2half2_rn(0.5f);
+        const float2 a = __half22float2(__hmul2(*reinterpret_cast<const __half2*>(&h01), half));
+        const float2 b = __half22float2(__hmul2(*reinterpret_cast<const __half2*>(&h23), half));
+        v[0] = a.x; v[1] = a.y; v[2] = b.x; v[3] = b.y;
         // bit 7 of a byte: its magnitude is all ones (the infinity) / its magnitude is zero and its sign is set (the NaN)
         const uint32_t mag = w & 0x7F7F7F7Fu;
         const uint32_t special = ((mag + 0x01010101u) | (~(mag + 0x7F7F7F7Fu) & w)) & 0x80808080u;
