@@ -41,6 +41,18 @@ def test_one_rank_nccl_group_equals_direct_calls():
             assert torch.equal(lp, direct) and torch.equal(opt.master, w) and torch.equal(opt.v, v)
             expect = capi.adam_update(wh, grad.cpu().numpy(), mh, vh, "bf16", "srf", 4, 10 + t, 0, 1e-3, 0.9, 0.99, 1e-8, t)
             gu.assert_codes_equal(lp, expect, "step %d" % t)
+        # the gradients written straight into the optimizer's persistent buffer, the gather left to be waited for later:
+        # same result, and a step takes no memory from the allocator
+        for t in range(4, 7):
+            grad = torch.randn(n, device="cuda", generator=g) * 1e-3
+            opt.grad_buffer().copy_(grad)
+            torch.cuda.synchronize()
+            allocated = torch.cuda.memory_allocated()
+            assert opt.step(opt.reduce_scatter_grad(), wait=False) is None
+            torch.cuda.synchronize()
+            assert torch.cuda.memory_allocated() == allocated
+            direct = fbsr.fbsr_adam_update(w, grad, m, v, "bf16", "srf", 4, 10 + t, 0, 1e-3, 0.9, 0.99, 1e-8, t)
+            assert torch.equal(opt.lp, direct) and torch.equal(opt.master, w) and torch.equal(opt.m, m)
         # the collective itself, as step() issues it for more than one rank: in place, on bytes
         own = opt.lp_padded[: opt.shard_len]
         before = opt.lp_padded.clone()
