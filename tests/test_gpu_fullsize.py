@@ -215,3 +215,42 @@ def test_small_update_accumulation_full_size(variant):
             assert moved == 0.0
     chk.report("accumulation %s, 20 of 1000 steps x 3 draw widths x 2^24" % variant)
     assert chk.fraction > 0.2
+
+
+@pytest.mark.parametrize("fmt,variant,k,data", [("bf16", "srf", 2, "sweep"), ("fp16", "src", 3, "sweep"), ("e4m3", "srf", 3, "fp8act")])
+def test_statistics_full_size(fmt, variant, k, data):
+    """The fused error statistics at the benchmark's sizes: counts equal and binary64 sums within 1e-9 of the oracle's
+    over every element (the oracle's per-piece totals added with an exact sum), codes included."""
+    import math
+    import threading
+    if data == "sweep":
+        x, scale = workloads.bandwidth_sweep(1 << 28, seed=1234, device="cuda"), 1.0
+    else:
+        x, scale = workloads.fp8_activations(fmt, device="cuda")
+    n = x.numel()
+    codes, st, _, _ = fbsr.fbsr_round_stats(x, fmt, variant, k, seed=1234, offset=0, scale=scale)
+    again = fbsr.fbsr_round_stats(x, fmt, variant, k, seed=1234, offset=0, scale=scale)[1]
+    assert again == st                                   # reproducible bit for bit
+    x_pin, xh = gu.pinned_like(x)
+    x_pin.copy_(x)
+    c_pin, ch = gu.pinned_like(codes)
+    c_pin.copy_(codes)
+    torch.cuda.synchronize()
+    pieces, lock = [], threading.Lock()
+
+    def piece(a, b):
+        ecodes, est, _, _ = capi.fbsr_round_stats(xh[a:b], fmt, variant, k, seed=1234, offset=a, scale=scale)
+        with lock:
+            pieces.append(est)
+        return gu.first_difference(ch[a:b], ecodes, a, "%s %s k=%d statistics codes" % (fmt, variant, k))
+
+    chk = gu.WholeTensorChecker(budget_s=120)
+    chk.run(n, piece)
+    chk.report("statistics %s %s k=%d, 2^%d elements" % (fmt, variant, k, n.bit_length() - 1))
+    assert chk.fraction == 1.0                           # totals need every piece
+    for key in ("n_finite", "n_up", "n_nan", "n_inf", "n_sat"):
+        assert st[key] == sum(p[key] for p in pieces), key
+    sum_abs = math.fsum(p["sum_abs_e"] for p in pieces)
+    for key in ("sum_e", "sum_e2", "sum_signed_e", "sum_abs_e"):
+        want = math.fsum(p[key] for p in pieces)
+        assert abs(st[key] - want) <= 1e-9 * max(abs(want), 1e-3 * sum_abs), (key, st[key], want)
